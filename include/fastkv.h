@@ -1,0 +1,180 @@
+/*
+ * fastkv.h -- C ABI of the B200 (sm_100a) FastKV token-saliency selection path.
+ *
+ * One layer's work is four calls on one CUDA stream:
+ *
+ *   fastkv_score       window-query saliency scores          (Eq. 1, Eq. 2, Sec. 4.2)
+ *   fastkv_select_kv   per-KV-group top-k   (KVCompress)      (App. B.1, Alg. 1)
+ *   fastkv_select_tsp  layer-level top-k    (HiddenCompress)  (App. B.1, Sec. 4.2)
+ *   fastkv_compact     gather of the kept K/V rows, hidden states and position ids
+ *                                                             (Alg. 1: C <- update(K, V); x)
+ *
+ * Conventions
+ *   - Every function returns a fastkv_status; nothing throws or aborts.
+ *   - Unless a parameter says HOST, every data pointer is DEVICE memory owned by the
+ *     caller.  The library allocates no device memory, keeps no pointer after the
+ *     enqueued work has run, and does not synchronise (fastkv_device_status and
+ *     fastkv_layer_host excepted).  Work is ordered on `stream` (a cudaStream_t
+ *     passed as void*; NULL is the legacy default stream).
+ *   - bf16 tensors are passed as void*; the innermost dimension is contiguous and
+ *     strides are counted in elements.
+ *   - Sequences of a batch are packed along the token axis: sequence b owns rows
+ *     cu_seqlens[b] .. cu_seqlens[b+1]-1, L_b = cu_seqlens[b+1]-cu_seqlens[b].
+ *     Token indices produced and consumed by the library are sequence-local.
+ *   - Inputs must be finite.  With NaN/Inf inputs the index sets are unspecified
+ *     (but in range).
+ */
+#ifndef FASTKV_H_
+#define FASTKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum fastkv_status {
+  FASTKV_OK = 0,
+  FASTKV_ERR_INVALID_ARG = 1,   /* NULL where a pointer is required, bad sizes, k out of range ...  */
+  FASTKV_ERR_UNSUPPORTED = 2,   /* valid but not built: head_dim, G*w, alignment, device generation */
+  FASTKV_ERR_WORKSPACE = 3,     /* workspace NULL, misaligned or smaller than fastkv_workspace_bytes */
+  FASTKV_ERR_CUDA = 4,          /* a CUDA call failed; fastkv_last_error() has the text             */
+  FASTKV_ERR_DEVICE_TIMEOUT = 5,/* a bounded device-side wait gave up (fastkv_device_status only)   */
+  FASTKV_ERR_DEVICE_INDEX = 6   /* an index handed to fastkv_compact was out of range; row skipped  */
+} fastkv_status;
+
+enum { FASTKV_POOL_AVG = 0, FASTKV_POOL_MAX = 1 };
+enum { FASTKV_GROUP_THEN_POOL = 0, FASTKV_POOL_THEN_GROUP = 1 };
+enum { FASTKV_Q_FULL = 0, FASTKV_Q_WINDOW = 1 };
+
+/*
+ * Problem statement of one layer (Sec. 4.2, App. B.1): N_I = L_b prompt tokens per
+ * sequence, N_obs = window, H = n_q_heads, key/value groups of G = H / n_kv_heads heads
+ * (query head h reads KV head h / G).
+ */
+typedef struct fastkv_shape {
+  int32_t batch;            /* B >= 1                                                         */
+  int32_t total_len;        /* sum of L_b: rows of the packed k / v / hidden / pos tensors   */
+  int32_t max_len;          /* max L_b (HOST knowledge used for grid sizing)                  */
+  int32_t n_q_heads;
+  int32_t n_kv_heads;
+  int32_t head_dim;         /* 64 or 128                                                      */
+  int32_t hidden_dim;       /* multiple of 8; only used by fastkv_compact                     */
+  int32_t window;           /* w = N_obs (paper: 8); G*w <= 64                                */
+  int32_t pool_kernel;      /* odd, 1..63 (paper: 7)                                          */
+  int32_t pool_mode;        /* FASTKV_POOL_AVG | FASTKV_POOL_MAX                              */
+  int32_t agg_order;        /* FASTKV_GROUP_THEN_POOL: pool the group-summed score;
+                               FASTKV_POOL_THEN_GROUP: pool per query head (Eq. 1), then sum
+                               within the group (App. B.1).  Identical for AVG up to rounding */
+  int32_t force_window;     /* 1: the last w positions are always kept and are not ranked
+                               (Sec. 4.2); 0: plain top-k over all positions                  */
+  int32_t q_layout;         /* FASTKV_Q_FULL: q has total_len rows, the library reads rows
+                               cu_seqlens[b+1]-w .. cu_seqlens[b+1]-1;
+                               FASTKV_Q_WINDOW: q has batch*w rows, sequence b at rows b*w..  */
+  float softmax_scale;      /* 0 => 1/sqrt(head_dim)                                          */
+  const int32_t* cu_seqlens;/* DEVICE int32[B+1], or NULL when B == 1 (then L = total_len)    */
+  int64_t q_stride_tok, q_stride_head;   /* elements; multiples of 8                          */
+  int64_t k_stride_tok, k_stride_head;
+  int64_t v_stride_tok, v_stride_head;
+  int64_t hidden_stride_tok;
+} fastkv_shape;
+
+/*
+ * How many positions each sequence keeps.  Either the same k for every sequence
+ * (k > 0, cu_k == NULL; sequence b writes outputs at offset b*k, total = B*k), or a
+ * DEVICE int32[B+1] array of output offsets (k_b = cu_k[b+1]-cu_k[b]) whose last entry
+ * the caller repeats on the host in `total`.  With force_window, w <= k_b <= L_b;
+ * otherwise 1 <= k_b <= L_b.  The uniform form is validated on the host against
+ * max_len only when B == 1; per-sequence violations clamp on the device and raise
+ * FASTKV_ERR_DEVICE_INDEX in the status word.
+ */
+typedef struct fastkv_budget {
+  int32_t k;
+  int32_t total;
+  const int32_t* cu_k;
+} fastkv_budget;
+
+/* Bytes of workspace needed by the calls below for this shape (a multiple of 256). */
+int fastkv_workspace_bytes(const fastkv_shape* shape, size_t* bytes);
+
+/*
+ * Saliency scores (Eq. 1 and Eq. 2; Sec. 4.2).  For each sequence, query head h and window
+ * row j (query position t_j = L-w+j) the causal softmax attention row over keys 0..t_j is
+ * formed, summed over the window, aggregated over each KV group and pooled along the
+ * sequence (kernel `pool_kernel`, stride 1, same length; AVG zero-pads and divides by the
+ * kernel size, MAX ignores out-of-range positions):
+ *   scores_kv [n_kv_heads, total_len] fp32   group-wise score used by KVCompress
+ *   scores_tsp[total_len] fp32 or NULL       sum over all heads (Eq. 2 up to the factor 1/H)
+ * Sums replace the paper's means; rankings are unchanged.
+ * q, k: bf16.  workspace: >= fastkv_workspace_bytes, 256-byte aligned; it also holds the
+ * device status word, so pass the same workspace to the other calls of the layer.
+ */
+int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float* scores_kv,
+                 float* scores_tsp, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * KVCompress selection (App. B.1): for every sequence and KV head, the k_b positions with the
+ * largest scores_kv, ties to the lower index; with force_window the last w positions are
+ * always kept and only the prefix is ranked.  idx_kv is int32 [n_kv_heads, budget.total],
+ * sequence-local, strictly ascending within each (head, sequence) segment.
+ */
+int fastkv_select_kv(const fastkv_shape* shape, const float* scores_kv, const fastkv_budget* budget,
+                     int32_t* idx_kv, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * HiddenCompress selection (App. B.1, Sec. 4.2): the same rule applied once per sequence to
+ * the layer-level score.  idx_tsp is int32 [budget.total].
+ */
+int fastkv_select_tsp(const fastkv_shape* shape, const float* scores_tsp, const fastkv_budget* budget,
+                      int32_t* idx_tsp, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Compaction (Alg. 1: C <- update(K, V); reduced hidden states x).  Byte copies:
+ *   k_out[g, j, :]   = k[cu_seqlens[b] + idx_kv[g, j], g, :]     [n_kv_heads, kv.total, head_dim]
+ *   v_out likewise                                               (v, v_out may both be NULL)
+ *   hidden_out[j, :] = hidden[cu_seqlens[b] + idx_tsp[j], :]     [tsp.total, hidden_dim]
+ *   pos_out[j]       = pos_ids[cu_seqlens[b] + idx_tsp[j]]       [tsp.total] int32
+ * where b is the sequence that owns output slot j.  Pass idx_tsp == NULL on layers without
+ * Token-Selective Propagation; hidden/hidden_out and pos_ids/pos_out may each be NULL.
+ * An index outside [0, L_b) is skipped and reported through the status word.
+ */
+int fastkv_compact(const fastkv_shape* shape, const int32_t* idx_kv, const fastkv_budget* kv,
+                   const int32_t* idx_tsp, const fastkv_budget* tsp, const void* k, const void* v,
+                   const void* hidden, const int32_t* pos_ids, void* k_out, void* v_out,
+                   void* hidden_out, int32_t* pos_out, void* workspace, size_t workspace_bytes,
+                   void* stream);
+
+/*
+ * Synchronises `stream`, then copies the device status word of `workspace` to the HOST
+ * integers *status (a fastkv_status) and *site (which wait or check raised it; 0 if none).
+ */
+int fastkv_device_status(const void* workspace, void* stream, int32_t* status, int32_t* site);
+
+/*
+ * One whole layer step from HOST buffers (the end-to-end path of the bench): copies q, k, v,
+ * hidden, pos_ids (HOST, pinned for full speed) into `arena` (DEVICE, caller-owned, at least
+ * fastkv_layer_host_arena_bytes), runs score -> select_kv -> select_tsp -> compact on `stream`,
+ * copies idx_kv, idx_tsp, k_out, v_out, hidden_out, pos_out back to the HOST outputs and
+ * synchronises.  B == 1 or uniform budgets only (budget.cu_k must be NULL); shape->cu_seqlens,
+ * if given, is a HOST array here.  k_tsp == 0 skips the TSP part.
+ */
+int fastkv_layer_host_arena_bytes(const fastkv_shape* shape, int32_t k_kv, int32_t k_tsp,
+                                  size_t* bytes);
+int fastkv_layer_host(const fastkv_shape* shape, int32_t k_kv, int32_t k_tsp, const void* q,
+                      const void* k, const void* v, const void* hidden, const int32_t* pos_ids,
+                      int32_t* idx_kv, int32_t* idx_tsp, void* k_out, void* v_out,
+                      void* hidden_out, int32_t* pos_out, void* arena, size_t arena_bytes,
+                      void* stream);
+
+/* Text for a fastkv_status; static storage. */
+const char* fastkv_status_string(int status);
+/* Text of the last FASTKV_ERR_CUDA / argument failure on the calling thread; static storage. */
+const char* fastkv_last_error(void);
+/* Number of kernels the library has launched from this process (for launch accounting). */
+int64_t fastkv_kernel_launches(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FASTKV_H_ */

@@ -1,0 +1,474 @@
+// C ABI of the FastKV selection path: argument validation, workspace carving, TMA descriptor
+// encoding and kernel launches.  Declarations and contracts live in include/fastkv.h.
+#include <atomic>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "compact.cuh"
+#include "score.cuh"
+#include "select.cuh"
+
+namespace fastkv {
+namespace {
+
+thread_local char g_last_error[512] = "";
+std::atomic<long long> g_launches{0};
+
+int fail(int status, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_last_error, sizeof g_last_error, fmt, ap);
+  va_end(ap);
+  return status;
+}
+
+int cuda_fail(cudaError_t e, const char* what) {
+  return fail(FASTKV_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int npad_for(int n_rows) { return n_rows <= 32 ? 32 : 64; }
+
+// ---- workspace layout --------------------------------------------------------------------------
+struct Layout {
+  int npad, tiles_per_cta, max_ranges;
+  long long ld_logits;
+  size_t off_counters, off_final, off_partial, off_logits, bytes, zero_bytes;
+};
+
+Layout make_layout(const fastkv_shape& s) {
+  Layout l;
+  const int G = s.n_q_heads / s.n_kv_heads;
+  l.npad = npad_for(G * s.window);
+  const long long max_tiles = (static_cast<long long>(s.max_len) + 127) / 128;
+  // about four waves of two co-resident CTAs per SM on a 148-SM part, at least two tiles per CTA
+  long long tpc = (max_tiles * s.n_kv_heads * s.batch + 1183) / 1184;
+  if (tpc < 2) tpc = 2;
+  if (tpc > 32) tpc = 32;
+  l.tiles_per_cta = static_cast<int>(tpc);
+  l.max_ranges = static_cast<int>((max_tiles + tpc - 1) / tpc);
+  if (l.max_ranges < 1) l.max_ranges = 1;
+  l.ld_logits = static_cast<long long>(round_up(static_cast<size_t>(s.total_len), 64));
+  size_t off = sizeof(WorkspaceHeader);
+  l.off_counters = off;
+  off += round_up(sizeof(int) * s.batch * s.n_kv_heads, 256);
+  l.zero_bytes = off;                       // header + counters are cleared by fastkv_score
+  l.off_final = off;
+  off += round_up(sizeof(float2) * s.batch * s.n_kv_heads * l.npad, 256);
+  l.off_partial = off;
+  off += round_up(sizeof(float2) * static_cast<size_t>(s.batch) * s.n_kv_heads * l.max_ranges * l.npad, 256);
+  l.off_logits = off;
+  off += round_up(sizeof(float) * static_cast<size_t>(s.n_kv_heads) * l.npad * l.ld_logits, 256);
+  l.bytes = off;
+  return l;
+}
+
+// ---- validation ---------------------------------------------------------------------------------
+int check_shape(const fastkv_shape* s, bool for_score) {
+  if (s == nullptr) return fail(FASTKV_ERR_INVALID_ARG, "shape is NULL");
+  if (s->batch < 1) return fail(FASTKV_ERR_INVALID_ARG, "batch must be >= 1");
+  if (s->total_len < 1 || s->max_len < 1 || s->max_len > s->total_len)
+    return fail(FASTKV_ERR_INVALID_ARG, "need 1 <= max_len <= total_len");
+  if (s->batch > 1 && s->cu_seqlens == nullptr)
+    return fail(FASTKV_ERR_INVALID_ARG, "cu_seqlens is required when batch > 1");
+  if (s->batch == 1 && s->max_len != s->total_len)
+    return fail(FASTKV_ERR_INVALID_ARG, "batch == 1 needs max_len == total_len");
+  if (s->n_kv_heads < 1 || s->n_q_heads < 1 || s->n_q_heads % s->n_kv_heads != 0)
+    return fail(FASTKV_ERR_INVALID_ARG, "n_q_heads must be a positive multiple of n_kv_heads");
+  if (s->window < 1) return fail(FASTKV_ERR_INVALID_ARG, "window must be >= 1");
+  if (s->batch == 1 && s->window > s->total_len)
+    return fail(FASTKV_ERR_INVALID_ARG, "window exceeds the sequence length");
+  if (s->force_window != 0 && s->force_window != 1)
+    return fail(FASTKV_ERR_INVALID_ARG, "force_window must be 0 or 1");
+  if (!for_score) return FASTKV_OK;
+  if (s->pool_kernel < 1 || (s->pool_kernel & 1) == 0)
+    return fail(FASTKV_ERR_INVALID_ARG, "pool_kernel must be odd and >= 1");
+  if (s->pool_kernel > 63) return fail(FASTKV_ERR_UNSUPPORTED, "pool_kernel > 63 is not built");
+  if (s->pool_mode != FASTKV_POOL_AVG && s->pool_mode != FASTKV_POOL_MAX)
+    return fail(FASTKV_ERR_INVALID_ARG, "unknown pool_mode");
+  if (s->agg_order != FASTKV_GROUP_THEN_POOL && s->agg_order != FASTKV_POOL_THEN_GROUP)
+    return fail(FASTKV_ERR_INVALID_ARG, "unknown agg_order");
+  if (s->q_layout != FASTKV_Q_FULL && s->q_layout != FASTKV_Q_WINDOW)
+    return fail(FASTKV_ERR_INVALID_ARG, "unknown q_layout");
+  if (!(s->softmax_scale >= 0.0f) || std::isinf(s->softmax_scale))
+    return fail(FASTKV_ERR_INVALID_ARG, "softmax_scale must be finite and >= 0");
+  if (s->head_dim != 64 && s->head_dim != 128)
+    return fail(FASTKV_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+  const int n_rows = s->n_q_heads / s->n_kv_heads * s->window;
+  if (n_rows > 64) return fail(FASTKV_ERR_UNSUPPORTED, "G * window > 64 is not built");
+  if (s->n_q_heads / s->n_kv_heads > 256 || s->window > 256)
+    return fail(FASTKV_ERR_UNSUPPORTED, "TMA box limit: G and window must be <= 256");
+  if (s->q_stride_tok % 8 || s->q_stride_head % 8 || s->k_stride_tok % 8 || s->k_stride_head % 8)
+    return fail(FASTKV_ERR_UNSUPPORTED, "q/k strides must be multiples of 8 elements (16 bytes)");
+  if (s->q_stride_head < s->head_dim || s->k_stride_head < s->head_dim ||
+      s->q_stride_tok < s->head_dim || s->k_stride_tok < s->head_dim)
+    return fail(FASTKV_ERR_INVALID_ARG, "q/k strides are smaller than head_dim");
+  return FASTKV_OK;
+}
+
+int check_workspace(const void* ws, size_t ws_bytes, size_t need) {
+  if (ws == nullptr) return fail(FASTKV_ERR_WORKSPACE, "workspace is NULL");
+  if (reinterpret_cast<uintptr_t>(ws) % 256) return fail(FASTKV_ERR_WORKSPACE, "workspace must be 256-byte aligned");
+  if (ws_bytes < need) return fail(FASTKV_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", ws_bytes, need);
+  return FASTKV_OK;
+}
+
+int check_budget(const fastkv_shape* s, const fastkv_budget* b, const char* name) {
+  if (b == nullptr) return fail(FASTKV_ERR_INVALID_ARG, "%s budget is NULL", name);
+  const int w = s->force_window ? s->window : 0;
+  if (b->cu_k == nullptr) {
+    if (b->k < 1 || b->k < w) return fail(FASTKV_ERR_INVALID_ARG, "%s: k must be >= max(1, window)", name);
+    if (b->k > s->max_len) return fail(FASTKV_ERR_INVALID_ARG, "%s: k exceeds the sequence length", name);
+    if (static_cast<long long>(b->k) * s->batch != b->total)
+      return fail(FASTKV_ERR_INVALID_ARG, "%s: total must equal batch * k", name);
+  } else {
+    if (b->total < 1) return fail(FASTKV_ERR_INVALID_ARG, "%s: total must be >= 1", name);
+  }
+  return FASTKV_OK;
+}
+
+// ---- TMA descriptors ------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 tensor [rows][heads][dim] with element strides; box = box_rows x box_heads x 64 columns
+int encode_bf16_3d(CUtensorMap* map, const void* base, int dim, int heads, long long rows,
+                   long long stride_head, long long stride_tok, int box_heads, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return fail(FASTKV_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  if (reinterpret_cast<uintptr_t>(base) % 16) return fail(FASTKV_ERR_UNSUPPORTED, "tensor base must be 16-byte aligned");
+  cuuint64_t dims[3] = {static_cast<cuuint64_t>(dim), static_cast<cuuint64_t>(heads), static_cast<cuuint64_t>(rows)};
+  cuuint64_t strides[2] = {static_cast<cuuint64_t>(stride_head) * 2, static_cast<cuuint64_t>(stride_tok) * 2};
+  cuuint32_t box[3] = {64, static_cast<cuuint32_t>(box_heads), static_cast<cuuint32_t>(box_rows)};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(FASTKV_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
+  return FASTKV_OK;
+}
+
+int check_device() {
+  static int ok = -1;
+  if (ok < 0) {
+    int dev = 0, major = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+    ok = (major == 10) ? 1 : 0;
+  }
+  if (!ok) return fail(FASTKV_ERR_UNSUPPORTED, "this library is built for sm_100a (B200) only");
+  return FASTKV_OK;
+}
+
+}  // namespace
+}  // namespace fastkv
+
+using namespace fastkv;
+
+extern "C" {
+
+int fastkv_workspace_bytes(const fastkv_shape* shape, size_t* bytes) {
+  int rc = check_shape(shape, true);
+  if (rc) return rc;
+  if (bytes == nullptr) return fail(FASTKV_ERR_INVALID_ARG, "bytes is NULL");
+  *bytes = make_layout(*shape).bytes;
+  return FASTKV_OK;
+}
+
+int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float* scores_kv,
+                 float* scores_tsp, void* workspace, size_t workspace_bytes, void* stream_) {
+  int rc = check_shape(shape, true);
+  if (rc) return rc;
+  if (q == nullptr || k == nullptr || scores_kv == nullptr)
+    return fail(FASTKV_ERR_INVALID_ARG, "q, k and scores_kv are required");
+  const Layout lay = make_layout(*shape);
+  if ((rc = check_workspace(workspace, workspace_bytes, lay.bytes))) return rc;
+  if ((rc = check_device())) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const fastkv_shape& s = *shape;
+  const int G = s.n_q_heads / s.n_kv_heads;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+
+  CUtensorMap tmap_k, tmap_q;
+  if ((rc = encode_bf16_3d(&tmap_k, k, s.head_dim, s.n_kv_heads, s.total_len, s.k_stride_head,
+                           s.k_stride_tok, 1, 128)))
+    return rc;
+  const long long q_rows = s.q_layout == FASTKV_Q_WINDOW ? static_cast<long long>(s.batch) * s.window : s.total_len;
+  if ((rc = encode_bf16_3d(&tmap_q, q, s.head_dim, s.n_q_heads, q_rows, s.q_stride_head, s.q_stride_tok,
+                           G, s.window)))
+    return rc;
+
+  cudaError_t e = cudaMemsetAsync(ws, 0, lay.zero_bytes, stream);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace header)");
+
+  ScoreParams sp;
+  sp.batch = s.batch; sp.total_len = s.total_len; sp.n_kv_heads = s.n_kv_heads; sp.group = G;
+  sp.window = s.window; sp.n_rows = G * s.window; sp.q_layout = s.q_layout;
+  sp.tiles_per_cta = lay.tiles_per_cta; sp.max_ranges = lay.max_ranges;
+  const float scale = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / std::sqrt(static_cast<float>(s.head_dim));
+  sp.scale_log2 = scale * 1.4426950408889634f;
+  sp.cu_seqlens = s.batch > 1 || s.cu_seqlens ? s.cu_seqlens : nullptr;
+  sp.logits = reinterpret_cast<float*>(ws + lay.off_logits);
+  sp.ld_logits = lay.ld_logits;
+  sp.partial = reinterpret_cast<float2*>(ws + lay.off_partial);
+  sp.final_stats = reinterpret_cast<float2*>(ws + lay.off_final);
+  sp.counters = reinterpret_cast<int*>(ws + lay.off_counters);
+  sp.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+  dim3 grid(s.n_kv_heads, lay.max_ranges, s.batch);
+  e = launch_score_logits(s.head_dim, lay.npad, tmap_k, tmap_q, sp, grid, stream);
+  if (e != cudaSuccess) return cuda_fail(e, "score_logits_kernel launch");
+  ++g_launches;
+
+  PoolParams pp;
+  pp.total_len = s.total_len; pp.n_kv_heads = s.n_kv_heads; pp.group = G; pp.window = s.window;
+  pp.npad = lay.npad; pp.pool_kernel = s.pool_kernel; pp.pool_mode = s.pool_mode; pp.agg_order = s.agg_order;
+  pp.cu_seqlens = sp.cu_seqlens; pp.logits = sp.logits; pp.ld_logits = lay.ld_logits;
+  pp.final_stats = sp.final_stats; pp.scores_kv = scores_kv; pp.ld_scores = s.total_len;
+  pp.scores_tsp = scores_tsp;
+  if (score_pool_smem_bytes(pp) > 200 * 1024)
+    return fail(FASTKV_ERR_UNSUPPORTED, "heads x pool halo do not fit the pooling kernel's shared memory");
+  e = launch_score_pool(pp, s.max_len, s.batch, stream);
+  if (e != cudaSuccess) return cuda_fail(e, "score_pool_kernel launch");
+  ++g_launches;
+  return FASTKV_OK;
+}
+
+static int select_common(const fastkv_shape* shape, const float* scores, const fastkv_budget* budget,
+                         int32_t* idx, int n_rows, void* workspace, size_t workspace_bytes, void* stream_,
+                         const char* name) {
+  int rc = check_shape(shape, false);
+  if (rc) return rc;
+  if (scores == nullptr || idx == nullptr) return fail(FASTKV_ERR_INVALID_ARG, "%s: scores and idx are required", name);
+  if ((rc = check_budget(shape, budget, name))) return rc;
+  if ((rc = check_workspace(workspace, workspace_bytes, sizeof(WorkspaceHeader)))) return rc;
+  if ((rc = check_device())) return rc;
+  SelectParams p;
+  p.scores = scores; p.ld_scores = shape->total_len; p.idx = idx; p.ld_idx = budget->total;
+  p.cu_seqlens = shape->cu_seqlens; p.cu_k = budget->cu_k; p.k_uniform = budget->k;
+  p.total_len = shape->total_len; p.window = shape->window; p.force_window = shape->force_window;
+  p.hdr = static_cast<WorkspaceHeader*>(workspace);
+  cudaError_t e = launch_select(p, n_rows, shape->batch, static_cast<cudaStream_t>(stream_));
+  if (e != cudaSuccess) return cuda_fail(e, "select_topk_kernel launch");
+  ++g_launches;
+  return FASTKV_OK;
+}
+
+int fastkv_select_kv(const fastkv_shape* shape, const float* scores_kv, const fastkv_budget* budget,
+                     int32_t* idx_kv, void* workspace, size_t workspace_bytes, void* stream) {
+  return select_common(shape, scores_kv, budget, idx_kv, shape ? shape->n_kv_heads : 0, workspace,
+                       workspace_bytes, stream, "select_kv");
+}
+
+int fastkv_select_tsp(const fastkv_shape* shape, const float* scores_tsp, const fastkv_budget* budget,
+                      int32_t* idx_tsp, void* workspace, size_t workspace_bytes, void* stream) {
+  return select_common(shape, scores_tsp, budget, idx_tsp, 1, workspace, workspace_bytes, stream, "select_tsp");
+}
+
+int fastkv_compact(const fastkv_shape* shape, const int32_t* idx_kv, const fastkv_budget* kv,
+                   const int32_t* idx_tsp, const fastkv_budget* tsp, const void* k, const void* v,
+                   const void* hidden, const int32_t* pos_ids, void* k_out, void* v_out,
+                   void* hidden_out, int32_t* pos_out, void* workspace, size_t workspace_bytes,
+                   void* stream_) {
+  int rc = check_shape(shape, false);
+  if (rc) return rc;
+  const fastkv_shape& s = *shape;
+  if ((rc = check_workspace(workspace, workspace_bytes, sizeof(WorkspaceHeader)))) return rc;
+  if ((k == nullptr) != (k_out == nullptr) || (v == nullptr) != (v_out == nullptr) ||
+      (hidden == nullptr) != (hidden_out == nullptr) || (pos_ids == nullptr) != (pos_out == nullptr))
+    return fail(FASTKV_ERR_INVALID_ARG, "compact: each source needs its destination and vice versa");
+  CompactParams cp;
+  memset(&cp, 0, sizeof cp);
+  cp.batch = s.batch; cp.total_len = s.total_len; cp.cu_seqlens = s.cu_seqlens;
+  cp.hdr = static_cast<WorkspaceHeader*>(workspace);
+  int n = 0;
+  if (k != nullptr || v != nullptr) {
+    if (idx_kv == nullptr) return fail(FASTKV_ERR_INVALID_ARG, "compact: idx_kv is required with k/v");
+    if ((rc = check_budget(shape, kv, "compact kv"))) return rc;
+    if (s.head_dim < 8 || s.head_dim % 8) return fail(FASTKV_ERR_UNSUPPORTED, "compact: head_dim must be a multiple of 8");
+    const void* src[2] = {k, v};
+    void* dst[2] = {k_out, v_out};
+    const long long st[2] = {s.k_stride_tok, s.v_stride_tok}, sh[2] = {s.k_stride_head, s.v_stride_head};
+    for (int t = 0; t < 2; ++t) {
+      if (src[t] == nullptr) continue;
+      if (st[t] % 8 || sh[t] % 8 || reinterpret_cast<uintptr_t>(src[t]) % 16 || reinterpret_cast<uintptr_t>(dst[t]) % 16)
+        return fail(FASTKV_ERR_UNSUPPORTED, "compact: k/v need 16-byte aligned bases and strides");
+      GatherJob& j = cp.job[n++];
+      j.src = static_cast<const uint8_t*>(src[t]); j.dst = static_cast<uint8_t*>(dst[t]);
+      j.idx = idx_kv; j.cu_k = kv->cu_k; j.k_uniform = kv->k; j.ld_idx = kv->total;
+      j.src_tok_bytes = st[t] * 2; j.src_head_bytes = sh[t] * 2;
+      j.heads = s.n_kv_heads; j.rows = kv->total; j.row_chunks = s.head_dim / 8;
+    }
+  }
+  if (hidden != nullptr || pos_ids != nullptr) {
+    if (idx_tsp == nullptr) return fail(FASTKV_ERR_INVALID_ARG, "compact: idx_tsp is required with hidden/pos_ids");
+    if ((rc = check_budget(shape, tsp, "compact tsp"))) return rc;
+    if (hidden != nullptr && (s.hidden_dim < 8 || s.hidden_dim % 8 || s.hidden_stride_tok % 8 ||
+                              s.hidden_stride_tok < s.hidden_dim ||
+                              reinterpret_cast<uintptr_t>(hidden) % 16 || reinterpret_cast<uintptr_t>(hidden_out) % 16))
+      return fail(FASTKV_ERR_UNSUPPORTED, "compact: hidden needs hidden_dim % 8 == 0 and 16-byte alignment");
+    GatherJob& j = cp.job[n++];
+    j.src = static_cast<const uint8_t*>(hidden); j.dst = static_cast<uint8_t*>(hidden_out);
+    j.idx = idx_tsp; j.cu_k = tsp->cu_k; j.k_uniform = tsp->k; j.ld_idx = tsp->total;
+    j.src_tok_bytes = s.hidden_stride_tok * 2; j.src_head_bytes = 0;
+    j.heads = 1; j.rows = tsp->total; j.row_chunks = hidden ? s.hidden_dim / 8 : 0;
+    j.pos_src = pos_ids; j.pos_dst = pos_out;
+  }
+  cp.n_jobs = n;
+  if (n == 0) return FASTKV_OK;
+  if ((rc = check_device())) return rc;
+  cudaError_t e = launch_compact(cp, static_cast<cudaStream_t>(stream_));
+  if (e != cudaSuccess) return cuda_fail(e, "compact_rows_kernel launch");
+  ++g_launches;
+  return FASTKV_OK;
+}
+
+int fastkv_device_status(const void* workspace, void* stream, int32_t* status, int32_t* site) {
+  if (workspace == nullptr || status == nullptr) return fail(FASTKV_ERR_INVALID_ARG, "workspace and status are required");
+  cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  int32_t words[2] = {0, 0};
+  e = cudaMemcpy(words, workspace, sizeof words, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status word)");
+  *status = words[0];
+  if (site) *site = words[1];
+  return FASTKV_OK;
+}
+
+// ---- host-buffer layer step -------------------------------------------------------------------------
+namespace {
+struct Arena {
+  size_t q, k, v, hidden, pos, cu, scores_kv, scores_tsp, idx_kv, idx_tsp, k_out, v_out, hidden_out, pos_out, ws;
+  size_t q_bytes, kv_bytes, hidden_bytes, ws_bytes, bytes;
+};
+Arena make_arena(const fastkv_shape& s, int k_kv, int k_tsp) {
+  Arena a;
+  size_t off = 0;
+  auto take = [&](size_t n) { size_t o = off; off += round_up(n, 256); return o; };
+  const size_t q_rows = s.q_layout == FASTKV_Q_WINDOW ? static_cast<size_t>(s.batch) * s.window : s.total_len;
+  a.q_bytes = q_rows * s.q_stride_tok * 2;
+  a.kv_bytes = static_cast<size_t>(s.total_len) * s.k_stride_tok * 2;
+  a.hidden_bytes = static_cast<size_t>(s.total_len) * s.hidden_stride_tok * 2;
+  a.q = take(a.q_bytes); a.k = take(a.kv_bytes); a.v = take(a.kv_bytes);
+  a.hidden = take(k_tsp ? a.hidden_bytes : 0); a.pos = take(k_tsp ? 4 * static_cast<size_t>(s.total_len) : 0);
+  a.cu = take(4 * (static_cast<size_t>(s.batch) + 1));
+  a.scores_kv = take(4 * static_cast<size_t>(s.n_kv_heads) * s.total_len);
+  a.scores_tsp = take(4 * static_cast<size_t>(s.total_len));
+  a.idx_kv = take(4 * static_cast<size_t>(s.n_kv_heads) * s.batch * k_kv);
+  a.idx_tsp = take(4 * static_cast<size_t>(s.batch) * k_tsp);
+  a.k_out = take(2 * static_cast<size_t>(s.n_kv_heads) * s.batch * k_kv * s.head_dim);
+  a.v_out = take(2 * static_cast<size_t>(s.n_kv_heads) * s.batch * k_kv * s.head_dim);
+  a.hidden_out = take(2 * static_cast<size_t>(s.batch) * k_tsp * s.hidden_dim);
+  a.pos_out = take(4 * static_cast<size_t>(s.batch) * k_tsp);
+  a.ws_bytes = make_layout(s).bytes;
+  a.ws = take(a.ws_bytes);
+  a.bytes = off;
+  return a;
+}
+}  // namespace
+
+int fastkv_layer_host_arena_bytes(const fastkv_shape* shape, int32_t k_kv, int32_t k_tsp, size_t* bytes) {
+  int rc = check_shape(shape, true);
+  if (rc) return rc;
+  if (bytes == nullptr || k_kv < 1 || k_tsp < 0) return fail(FASTKV_ERR_INVALID_ARG, "layer_host: bad k or NULL bytes");
+  *bytes = make_arena(*shape, k_kv, k_tsp).bytes;
+  return FASTKV_OK;
+}
+
+int fastkv_layer_host(const fastkv_shape* shape, int32_t k_kv, int32_t k_tsp, const void* q,
+                      const void* k, const void* v, const void* hidden, const int32_t* pos_ids,
+                      int32_t* idx_kv, int32_t* idx_tsp, void* k_out, void* v_out,
+                      void* hidden_out, int32_t* pos_out, void* arena, size_t arena_bytes,
+                      void* stream_) {
+  int rc = check_shape(shape, true);
+  if (rc) return rc;
+  if (k_kv < 1 || k_tsp < 0) return fail(FASTKV_ERR_INVALID_ARG, "layer_host: bad k");
+  if (!q || !k || !v || !idx_kv || !k_out || !v_out) return fail(FASTKV_ERR_INVALID_ARG, "layer_host: q, k, v and the kv outputs are required");
+  if (k_tsp && (!hidden || !pos_ids || !idx_tsp || !hidden_out || !pos_out))
+    return fail(FASTKV_ERR_INVALID_ARG, "layer_host: the TSP part needs hidden, pos_ids and their outputs");
+  const Arena a = make_arena(*shape, k_kv, k_tsp);
+  if ((rc = check_workspace(arena, arena_bytes, a.bytes))) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  uint8_t* d = static_cast<uint8_t*>(arena);
+  fastkv_shape s = *shape;
+  cudaError_t e;
+#define FASTKV_COPY(dst, src, n, kind)                                             \
+  if ((n) && (e = cudaMemcpyAsync(dst, src, n, kind, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync")
+  FASTKV_COPY(d + a.q, q, a.q_bytes, cudaMemcpyHostToDevice);
+  FASTKV_COPY(d + a.k, k, a.kv_bytes, cudaMemcpyHostToDevice);
+  FASTKV_COPY(d + a.v, v, a.kv_bytes, cudaMemcpyHostToDevice);
+  if (k_tsp) {
+    FASTKV_COPY(d + a.hidden, hidden, a.hidden_bytes, cudaMemcpyHostToDevice);
+    FASTKV_COPY(d + a.pos, pos_ids, 4 * static_cast<size_t>(s.total_len), cudaMemcpyHostToDevice);
+  }
+  if (shape->cu_seqlens) {
+    FASTKV_COPY(d + a.cu, shape->cu_seqlens, 4 * (static_cast<size_t>(s.batch) + 1), cudaMemcpyHostToDevice);
+    s.cu_seqlens = reinterpret_cast<const int32_t*>(d + a.cu);
+  }
+  float* scores_kv = reinterpret_cast<float*>(d + a.scores_kv);
+  float* scores_tsp = k_tsp ? reinterpret_cast<float*>(d + a.scores_tsp) : nullptr;
+  void* ws = d + a.ws;
+  if ((rc = fastkv_score(&s, d + a.q, d + a.k, scores_kv, scores_tsp, ws, a.ws_bytes, stream))) return rc;
+  fastkv_budget bkv = {k_kv, k_kv * s.batch, nullptr}, btsp = {k_tsp, k_tsp * s.batch, nullptr};
+  int32_t* d_idx_kv = reinterpret_cast<int32_t*>(d + a.idx_kv);
+  int32_t* d_idx_tsp = reinterpret_cast<int32_t*>(d + a.idx_tsp);
+  if ((rc = fastkv_select_kv(&s, scores_kv, &bkv, d_idx_kv, ws, a.ws_bytes, stream))) return rc;
+  if (k_tsp && (rc = fastkv_select_tsp(&s, scores_tsp, &btsp, d_idx_tsp, ws, a.ws_bytes, stream))) return rc;
+  if ((rc = fastkv_compact(&s, d_idx_kv, &bkv, k_tsp ? d_idx_tsp : nullptr, k_tsp ? &btsp : nullptr, d + a.k, d + a.v,
+                           k_tsp ? d + a.hidden : nullptr, k_tsp ? reinterpret_cast<const int32_t*>(d + a.pos) : nullptr,
+                           d + a.k_out, d + a.v_out, k_tsp ? d + a.hidden_out : nullptr,
+                           k_tsp ? reinterpret_cast<int32_t*>(d + a.pos_out) : nullptr, ws, a.ws_bytes, stream)))
+    return rc;
+  const size_t n_kv = static_cast<size_t>(s.n_kv_heads) * s.batch * k_kv;
+  FASTKV_COPY(idx_kv, d_idx_kv, 4 * n_kv, cudaMemcpyDeviceToHost);
+  FASTKV_COPY(k_out, d + a.k_out, 2 * n_kv * s.head_dim, cudaMemcpyDeviceToHost);
+  FASTKV_COPY(v_out, d + a.v_out, 2 * n_kv * s.head_dim, cudaMemcpyDeviceToHost);
+  if (k_tsp) {
+    const size_t n_t = static_cast<size_t>(s.batch) * k_tsp;
+    FASTKV_COPY(idx_tsp, d_idx_tsp, 4 * n_t, cudaMemcpyDeviceToHost);
+    FASTKV_COPY(hidden_out, d + a.hidden_out, 2 * n_t * s.hidden_dim, cudaMemcpyDeviceToHost);
+    FASTKV_COPY(pos_out, d + a.pos_out, 4 * n_t, cudaMemcpyDeviceToHost);
+  }
+#undef FASTKV_COPY
+  int32_t status = 0, site = 0;
+  if ((rc = fastkv_device_status(ws, stream, &status, &site))) return rc;
+  if (status != FASTKV_OK) return fail(status, "device status %d raised at site %d", status, site);
+  return FASTKV_OK;
+}
+
+const char* fastkv_status_string(int status) {
+  switch (status) {
+    case FASTKV_OK: return "ok";
+    case FASTKV_ERR_INVALID_ARG: return "invalid argument";
+    case FASTKV_ERR_UNSUPPORTED: return "unsupported configuration";
+    case FASTKV_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case FASTKV_ERR_CUDA: return "CUDA call failed";
+    case FASTKV_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
+    case FASTKV_ERR_DEVICE_INDEX: return "an index or budget was out of range on the device";
+    default: return "unknown status";
+  }
+}
+
+const char* fastkv_last_error(void) { return g_last_error; }
+
+int64_t fastkv_kernel_launches(void) { return g_launches.load(); }
+
+}  // extern "C"

@@ -1,0 +1,45 @@
+// Parameter blocks and launchers of the scoring kernels (see score.cu).
+#pragma once
+
+#include "common.cuh"
+
+namespace fastkv {
+
+constexpr int kPoolKeys = 256;      // positions produced by one CTA of the pooling kernel
+constexpr int kPoolThreads = 256;
+
+struct ScoreParams {
+  int batch, total_len, n_kv_heads, group, window;
+  int n_rows;                 // G * w query rows per KV head (columns of the accumulator)
+  int q_layout;
+  int tiles_per_cta;          // 128-key tiles handled by one CTA
+  int max_ranges;             // CTAs per (sequence, head) the partial-statistics array is sized for
+  float scale_log2;           // softmax scale times log2(e): logits are kept in log2 units
+  const int* cu_seqlens;      // device, may be null (single sequence)
+  float* logits;              // [Hkv][NPAD][ld_logits], masked entries hold -inf
+  long long ld_logits;
+  float2* partial;            // [B][Hkv][max_ranges][NPAD] per-CTA (max, sum of exp2)
+  float2* final_stats;        // [B][Hkv][NPAD] (row max, 1 / row sum)
+  int* counters;              // [B][Hkv] CTAs finished; zero before and after the kernel
+  WorkspaceHeader* hdr;
+};
+
+struct PoolParams {
+  int total_len, n_kv_heads, group, window, npad;
+  int pool_kernel, pool_mode, agg_order;
+  const int* cu_seqlens;
+  const float* logits;
+  long long ld_logits;
+  const float2* final_stats;
+  float* scores_kv;           // [Hkv][ld_scores]
+  long long ld_scores;
+  float* scores_tsp;          // [total_len] or null
+};
+
+cudaError_t launch_score_logits(int head_dim, int npad, const CUtensorMap& tmap_k,
+                                const CUtensorMap& tmap_q, const ScoreParams& p, dim3 grid,
+                                cudaStream_t stream);
+size_t score_pool_smem_bytes(const PoolParams& p);
+cudaError_t launch_score_pool(const PoolParams& p, int max_len, int batch, cudaStream_t stream);
+
+}  // namespace fastkv
