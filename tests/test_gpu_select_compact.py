@@ -117,7 +117,7 @@ def run_compact(lens, ks_kv, ks_tsp, Hkv, d, hidden, kbuf, vbuf, hbuf, pos, idx_
                 k_tok_stride=None, hidden_stride=None):
     total, Bn = sum(lens), len(lens)
     cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
-    d_cu = torch.from_numpy(cu).cuda() if ragged else None
+    d_cu = torch.from_numpy(cu).cuda() if (ragged or Bn > 1) else None
     shape = B.make_shape(total_len=total, n_q_heads=Hkv, n_kv_heads=Hkv, head_dim=d, hidden_dim=hidden, batch=Bn,
                          max_len=max(lens), cu_seqlens=d_cu, k_stride_tok=k_tok_stride, v_stride_tok=k_tok_stride,
                          hidden_stride_tok=hidden_stride)
