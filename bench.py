@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Benchmark of the FastKV score -> select -> compact layer step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One "step" is one pass of the whole hot path (fastkv_score, fastkv_select_kv, fastkv_select_tsp,
+fastkv_compact) over one layer of synthetic, seeded input.  The default workload is the
+Llama-3.1-8B-shaped layer at L = 131072 with Token-Selective Propagation (KV retention 10 %, TSP
+rate 20 %).  With N > 1 (torchrun, one rank per GPU) every rank runs its own layer of the same
+shape -- the path partitions over independent layers / requests, so there is no collective on the
+data path -- and the reported value is all ranks' tokens over the slowest rank's time.
+
+Prints one JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2502_01068_b200 import workloads as W  # noqa: E402
+
+METRIC = "context tokens/sec for score+select+compact, per layer"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def pick_workload(name: str) -> W.Workload:
+    table = {
+        "llama8b_128k_tsp_layer": W.llama8b_128k(),
+        "llama8b_8k": W.llama8b_8k(),
+        "llama8b_32k_tsp_layer": W.llama8b_32k_sweep(),
+        "llama8b_ragged": W.llama8b_ragged(),
+        "tiny": W.tiny(),
+    }
+    return table[name]
+
+
+def algorithmic_bytes(wl: W.Workload) -> dict:
+    """Bytes the step must move (each tensor read or written once): K streamed by the scoring, the
+    window queries, scores written and read, indices written and read, kept rows read and written."""
+    Hkv, d, hid = wl.n_kv_heads, wl.head_dim, wl.hidden_dim
+    total = wl.total_len
+    kkv = sum(wl.k_kv)
+    kt = sum(wl.k_tsp) if wl.k_tsp else 0
+    k_read = total * Hkv * d * 2
+    q_read = wl.batch * wl.window * wl.n_q_heads * d * 2
+    scores = 4 * (Hkv * total + (total if kt else 0))
+    idx = 4 * (Hkv * kkv + kt)
+    kv_rows = 2 * Hkv * kkv * d * 2
+    hid_rows = kt * (hid * 2 + 4)
+    return {
+        "score": k_read + q_read + scores,
+        "select": scores + idx,
+        "compact": idx + 2 * kv_rows + 2 * hid_rows,
+        "step_rw": k_read + q_read + 2 * scores + 2 * idx + 2 * kv_rows + 2 * hid_rows,
+        "step_min": k_read + q_read + 2 * scores + 2 * idx + kv_rows + hid_rows,
+    }
+
+
+def measured_peaks() -> dict:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "source": "measured (MEASURED_PEAKS.json)"}
+    return {"hbm_gbs": 6650.0, "source": "fallback (earlier measurement on this pool)"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.002):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake_slowdown",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if bit and (mask & bit):
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self) -> dict:
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2.0)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_baseline(wl: W.Workload, x: W.LayerInputs, budget_s: float = 20.0, max_reps: int = 3) -> dict:
+    """Times the fp64 oracle, as it stands, on this machine's host cores on the same layer."""
+    import oracle
+    from oracle.layer import layer_step
+    oracle.build()
+    reps, times = 0, []
+    t_all = time.perf_counter()
+    while reps < max_reps and (time.perf_counter() - t_all) < budget_s:
+        t0 = time.perf_counter()
+        layer_step(x.q_win, x.k, x.v, x.hidden, x.pos, x.cu_seqlens, wl.window, wl.pool_kernel, wl.k_kv,
+                   wl.k_tsp, pool_mode=wl.pool_mode)
+        times.append(time.perf_counter() - t0)
+        reps += 1
+    t = statistics.mean(times)
+    return {"value": wl.total_len / t, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "the whole layer (%d tokens), mean of %d run(s), %.2f s each" % (wl.total_len, reps, t)}
+
+
+def run_reference(args) -> None:
+    """--impl reference: the oracle is the reference arm (no reference implementation exists)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from oracle.layer import layer_step
+    oracle.build()
+    wl = pick_workload(args.workload)
+    x = W.make_layer(wl)
+    # each step is the whole layer; steps are capped so that the run ends within a few minutes
+    t0 = time.perf_counter()
+    layer_step(x.q_win, x.k, x.v, x.hidden, x.pos, x.cu_seqlens, wl.window, wl.pool_kernel, wl.k_kv, wl.k_tsp,
+               pool_mode=wl.pool_mode)
+    one = time.perf_counter() - t0
+    warm = max(0, min(args.warmup, int(20.0 / max(one, 1e-3)) - 1))
+    steps = max(1, min(args.steps, int(90.0 / max(one, 1e-3))))
+    for _ in range(warm):
+        layer_step(x.q_win, x.k, x.v, x.hidden, x.pos, x.cu_seqlens, wl.window, wl.pool_kernel, wl.k_kv,
+                   wl.k_tsp, pool_mode=wl.pool_mode)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        layer_step(x.q_win, x.k, x.v, x.hidden, x.pos, x.cu_seqlens, wl.window, wl.pool_kernel, wl.k_kv,
+                   wl.k_tsp, pool_mode=wl.pool_mode)
+    dt = (time.perf_counter() - t0) / steps
+    value = wl.total_len / dt
+    sample = "the whole layer per step; %d timed step(s) of %.2f s (requested %d)" % (steps, dt, args.steps)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "seq_lens": wl.seq_lens if wl.batch <= 8 else "ragged"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="llama8b_128k_tsp_layer")
+    ap.add_argument("--impl", default="fastkv", choices=["fastkv", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_2502_01068_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    warmup = max(3, args.warmup)
+    steps = max(1, args.steps)
+
+    wl = pick_workload(args.workload)
+    x = W.make_layer(wl, layer=rank)                      # each rank owns an independent layer
+    lens, Bn, total = wl.seq_lens, wl.batch, wl.total_len
+    tdev = lambda a: torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).cuda()
+    d_cu = tdev(x.cu_seqlens) if Bn > 1 else None
+    shape = B.make_shape(total_len=total, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim,
+                         hidden_dim=wl.hidden_dim, window=wl.window, pool_kernel=wl.pool_kernel,
+                         pool_mode=wl.pool_mode, batch=Bn, max_len=max(lens), cu_seqlens=d_cu)
+    q, k, v, hid, pos = tdev(x.q_win), tdev(x.k), tdev(x.v), tdev(x.hidden), tdev(x.pos)
+
+    def budget(ks):
+        if len(set(ks)) == 1:
+            return B.make_budget(int(ks[0]), batch=Bn), None
+        cu_k = tdev(np.concatenate([[0], np.cumsum(ks)]).astype(np.int32))
+        return B.make_budget(0, cu_k=cu_k, total=int(sum(ks))), cu_k
+
+    b_kv, _keep1 = budget(wl.k_kv)
+    b_tsp, _keep2 = budget(wl.k_tsp)
+    ws = torch.empty(B.fastkv_workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+    s_kv = torch.empty((wl.n_kv_heads, total), dtype=torch.float32, device="cuda")
+    s_tsp = torch.empty((total,), dtype=torch.float32, device="cuda")
+    idx_kv = torch.empty((wl.n_kv_heads, b_kv.total), dtype=torch.int32, device="cuda")
+    idx_tsp = torch.empty((b_tsp.total,), dtype=torch.int32, device="cuda")
+    k_out = torch.empty((wl.n_kv_heads, b_kv.total, wl.head_dim), dtype=torch.int16, device="cuda")
+    v_out = torch.empty_like(k_out)
+    hid_out = torch.empty((b_tsp.total, wl.hidden_dim), dtype=torch.int16, device="cuda")
+    pos_out = torch.empty((b_tsp.total,), dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step(events=None):
+        if events is not None:
+            events[0].record(stream)
+        B.fastkv_score(shape, q, k, s_kv, s_tsp, ws, stream)
+        if events is not None:
+            events[1].record(stream)
+        B.fastkv_select_kv(shape, s_kv, b_kv, idx_kv, ws, stream)
+        if events is not None:
+            events[2].record(stream)
+        B.fastkv_select_tsp(shape, s_tsp, b_tsp, idx_tsp, ws, stream)
+        if events is not None:
+            events[3].record(stream)
+        B.fastkv_compact(shape, idx_kv, b_kv, idx_tsp, b_tsp, k, v, hid, pos, k_out, v_out, hid_out, pos_out, ws,
+                         stream)
+        if events is not None:
+            events[4].record(stream)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    status, site = B.fastkv_device_status(ws)
+    if status != 0:
+        raise SystemExit("device status %d at site %d after warm-up" % (status, site))
+
+    # ---- timed region: K steps, device-timed, per-call events inside ---------------------------------
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
+    sampler = ClockSampler(local_rank)
+    launches0 = B.fastkv_kernel_launches()
+    barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    for i in range(steps):
+        step(ev[i])
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    launches = B.fastkv_kernel_launches() - launches0
+    total_ms = ev[0][0].elapsed_time(ev[-1][4])
+    call_ms = [statistics.mean(ev[i][c].elapsed_time(ev[i][c + 1]) for i in range(steps)) for c in range(4)]
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / steps
+    value = world * total / (ms_per_step * 1e-3)
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies timed) -------------
+    e2e = None
+    uniform = len(set(wl.k_kv)) == 1 and len(set(wl.k_tsp)) == 1
+    if uniform and args.e2e_steps > 0:
+        pin = lambda a: torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+        hq, hk, hv, hh, hp = pin(x.q_win), pin(x.k), pin(x.v), pin(x.hidden), pin(x.pos)
+        kk, kt = int(wl.k_kv[0]), int(wl.k_tsp[0])
+        o_idx_kv = torch.empty((wl.n_kv_heads, Bn * kk), dtype=torch.int32).pin_memory()
+        o_idx_tsp = torch.empty((Bn * kt,), dtype=torch.int32).pin_memory()
+        o_k = torch.empty((wl.n_kv_heads, Bn * kk, wl.head_dim), dtype=torch.int16).pin_memory()
+        o_v = torch.empty_like(o_k).pin_memory()
+        o_h = torch.empty((Bn * kt, wl.hidden_dim), dtype=torch.int16).pin_memory()
+        o_p = torch.empty((Bn * kt,), dtype=torch.int32).pin_memory()
+        hshape = B.make_shape(total_len=total, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads,
+                              head_dim=wl.head_dim, hidden_dim=wl.hidden_dim, window=wl.window,
+                              pool_kernel=wl.pool_kernel, pool_mode=wl.pool_mode, batch=Bn, max_len=max(lens),
+                              cu_seqlens=x.cu_seqlens if Bn > 1 else None)
+        arena = torch.empty(B.fastkv_layer_host_arena_bytes(hshape, kk, kt), dtype=torch.uint8, device="cuda")
+
+        def host_step():
+            B.fastkv_layer_host(hshape, kk, kt, hq, hk, hv, hh, hp, o_idx_kv, o_idx_tsp, o_k, o_v, o_h, o_p, arena,
+                                stream)
+
+        host_step()
+        barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            host_step()                                   # synchronises: outputs are on the host
+        e2e_s = (time.perf_counter() - t0) / args.e2e_steps
+        if world > 1:
+            import torch.distributed as dist
+            t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hh, hp))
+        d2h = sum(t.numel() * t.element_size() for t in (o_idx_kv, o_idx_tsp, o_k, o_v, o_h, o_p))
+        e2e = {"value": world * total / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": e2e_s * 1e3, "steps": args.e2e_steps}
+        if np.array_equal(o_idx_tsp.numpy(), idx_tsp.cpu().numpy()) is False:
+            raise SystemExit("host-buffer path and device path disagree on idx_tsp")
+
+    if rank != 0:
+        return
+    ab = algorithmic_bytes(wl)
+    peaks = measured_peaks()
+    compact_gbs = ab["compact"] / (call_ms[3] * 1e-3) / 1e9
+    step_gbs = ab["step_rw"] / (ms_per_step * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "seq_lens": lens, "k_kv": wl.k_kv, "k_tsp": wl.k_tsp,
+                   "n_q_heads": wl.n_q_heads, "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim,
+                   "hidden_dim": wl.hidden_dim, "window": wl.window, "pool_kernel": wl.pool_kernel,
+                   "l2": "inputs larger than L2 (K %.0f MB, hidden %.0f MB per step)" % (
+                       x.k.nbytes / 1e6, x.hidden.nbytes / 1e6)},
+        "clocks": clocks,
+        "gpu_launches": int(launches),
+        "e2e": e2e,
+        "roofline": {"bound": "hbm", "kernel": "compact_rows_kernel", "achieved": compact_gbs,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": compact_gbs / peaks["hbm_gbs"],
+                     "peak_source": peaks["source"], "algorithmic_bytes": ab["compact"], "traffic": None,
+                     "ms": call_ms[3]},
+        "step_roofline": {"bytes_rw": ab["step_rw"], "bytes_rows_once": ab["step_min"], "achieved_gbs": step_gbs,
+                          "frac_of_measured": step_gbs / peaks["hbm_gbs"],
+                          "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
+                          "rows_once_gbs": ab["step_min"] / (ms_per_step * 1e-3) / 1e9},
+        "calls_ms": {"fastkv_score": call_ms[0], "fastkv_select_kv": call_ms[1], "fastkv_select_tsp": call_ms[2],
+                     "fastkv_compact": call_ms[3]},
+        "calls_gbs": {"fastkv_score": ab["score"] / (call_ms[0] * 1e-3) / 1e9},
+    }
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"] = oracle_baseline(wl, x)
+    print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()
