@@ -167,6 +167,29 @@ int fastkv_layer_host(const fastkv_shape* shape, int32_t k_kv, int32_t k_tsp, co
                       void* hidden_out, int32_t* pos_out, void* arena, size_t arena_bytes,
                       void* stream);
 
+/*
+ * fastkv_score for callers that cannot allocate device memory (no counterpart in the paper:
+ * this is a deployment variant, not a step of the method).  Some callers have no workspace to
+ * give: a plug-in inside a serving process whose device allocator belongs to the host
+ * framework, code that runs where cudaMalloc is not permitted, a minimal C client without an
+ * allocator.  This entry point computes exactly what fastkv_score computes, with the scratch
+ * memory of the scoring kernels held in a fixed 16 MiB device array inside the library (so
+ * every GPU that loads the library carries those 16 MiB until the process exits).  It calls no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *   - Limit: fastkv_workspace_bytes(shape) must be <= 16 MiB (Llama-3.1-8B head shape: up to
+ *     16 000 tokens per call); larger shapes return FASTKV_ERR_WORKSPACE and launch nothing.
+ *   - The first call on each device looks up the array's device address (the device must be
+ *     current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the
+ *     words that must start at zero are cleared on `stream` by every call.  Two calls whose
+ *     GPU work overlaps (different streams, no ordering) race on it: serialise them.
+ *   - The device status word lives inside the array and is not exposed; waits on the device
+ *     stay bounded as in fastkv_score.
+ * q, k, scores_kv, scores_tsp, stream: as for fastkv_score.
+ */
+int fastkv_score_static(const fastkv_shape* shape, const void* q, const void* k, float* scores_kv,
+                        float* scores_tsp, void* stream);
+
 /* Text for a fastkv_status; static storage. */
 const char* fastkv_status_string(int status);
 /* Text of the last FASTKV_ERR_CUDA / argument failure on the calling thread; static storage. */

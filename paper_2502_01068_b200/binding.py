@@ -22,7 +22,8 @@ Q_FULL, Q_WINDOW = 0, 1
 
 EXPORTS = ["fastkv_workspace_bytes", "fastkv_score", "fastkv_select_kv", "fastkv_select_tsp",
            "fastkv_compact", "fastkv_device_status", "fastkv_layer_host_arena_bytes",
-           "fastkv_layer_host", "fastkv_status_string", "fastkv_last_error", "fastkv_kernel_launches"]
+           "fastkv_layer_host", "fastkv_score_static", "fastkv_status_string", "fastkv_last_error",
+           "fastkv_kernel_launches"]
 
 
 class FastKVError(RuntimeError):
@@ -78,7 +79,8 @@ def _load():
         lib.fastkv_status_string.restype = ctypes.c_char_p
         lib.fastkv_last_error.restype = ctypes.c_char_p
         lib.fastkv_kernel_launches.restype = ctypes.c_int64
-        for fn in EXPORTS[:8]:
+        lib.fastkv_score_static.argtypes = [ps, vp, vp, vp, vp, vp]
+        for fn in EXPORTS[:9]:
             getattr(lib, fn).restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -194,6 +196,14 @@ def fastkv_layer_host(shape: Shape, k_kv: int, k_tsp: int, q, k, v, hidden, pos_
                                      _p(hidden_out), _p(pos_out), _p(arena),
                                      arena.numel() * arena.element_size(), _stream(stream)),
            "fastkv_layer_host")
+
+
+def fastkv_score_static(shape: Shape, q, k, scores_kv, scores_tsp, stream=None) -> None:
+    """fastkv_score without a workspace argument: the scratch is a fixed 16 MiB array inside the
+    library, for callers that cannot allocate device memory.  Shapes that need more raise
+    FastKVError(ERR_WORKSPACE).  Calls on one device share the array: do not overlap them."""
+    _check(_load().fastkv_score_static(ctypes.byref(shape), _p(q), _p(k), _p(scores_kv), _p(scores_tsp),
+                                       _stream(stream)), "fastkv_score_static")
 
 
 def fastkv_status_string(status: int) -> str:

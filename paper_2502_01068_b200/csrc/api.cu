@@ -180,6 +180,11 @@ int check_device() {
 }
 
 }  // namespace
+
+// Lets the other translation units of the library leave their message where fastkv_last_error()
+// finds it.
+int report_error(int status, const char* text) { return fail(status, "%s", text); }
+
 }  // namespace fastkv
 
 using namespace fastkv;

@@ -31,6 +31,9 @@ enum Site : int {
   SITE_SELECT_BUDGET = 17,
 };
 
+// Records `text` as the calling thread's last error (see fastkv_last_error) and returns `status`.
+int report_error(int status, const char* text);
+
 __device__ __forceinline__ void raise_status(WorkspaceHeader* hdr, int status, int site) {
   if (hdr != nullptr && atomicCAS(&hdr->status, 0, status) == 0) hdr->site = site;
 }
