@@ -271,7 +271,7 @@ static int select_common(const fastkv_shape* shape, const float* scores, const f
   p.cu_seqlens = shape->cu_seqlens; p.cu_k = budget->cu_k; p.k_uniform = budget->k;
   p.total_len = shape->total_len; p.window = shape->window; p.force_window = shape->force_window;
   p.hdr = static_cast<WorkspaceHeader*>(workspace);
-  cudaError_t e = launch_select(p, n_rows, shape->batch, static_cast<cudaStream_t>(stream_));
+  cudaError_t e = launch_select(p, n_rows, shape->batch, shape->max_len, static_cast<cudaStream_t>(stream_));
   if (e != cudaSuccess) return cuda_fail(e, "select_topk_kernel launch");
   ++g_launches;
   return FASTKV_OK;

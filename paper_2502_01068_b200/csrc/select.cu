@@ -30,23 +30,31 @@ __device__ __forceinline__ uint32_t order_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-struct SelShared {
+struct alignas(16) SelShared {
   int hist[kBins * 32];          // lane-private digit counters: hist[bin * 32 + lane]
   int block_hist[2][kBins];      // this CTA's histogram, double-buffered by pass parity
+  int total_hist[kBins];         // the cluster's histogram of the current pass
   int warp_tot[2][kSelWarps];
-  int counts[2];                 // this CTA's (#above threshold, #equal to threshold)
+  alignas(8) int counts[2];      // this CTA's (#above threshold, #equal to threshold)
   int digit, k_rem;
 };
 
 }  // namespace
 
-template <int CLUSTER>
+// ITEMS > 0: every thread keeps its ITEMS candidates (converted once) in registers for all
+// passes; candidate (warp w, round r, lane l) of a CTA is c_begin + (w * ITEMS + r) * 32 + l, so
+// loads are coalesced and index order is (warp, round, lane).  ITEMS == 0: any chunk size, every
+// pass re-reads the scores (they are L2 resident).
+template <int CLUSTER, int ITEMS>
 __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const SelectParams p) {
   cg::cluster_group cluster = cg::this_cluster();
   __shared__ SelShared sh;
+  constexpr bool CACHED = ITEMS > 0;
+  constexpr int R = CACHED ? ITEMS : 1;
   const int rank = static_cast<int>(cluster.block_rank());
   const int row = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t lt_mask = (1u << lane) - 1u;
 
   const int row0 = p.cu_seqlens ? p.cu_seqlens[b] : 0;
   const int L = p.cu_seqlens ? p.cu_seqlens[b + 1] - row0 : p.total_len;
@@ -65,48 +73,76 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
   }
   const int n_cand = L - w;          // ranked positions: [0, n_cand)
   const int k_sel = k - w;           // how many of them are kept
-  // contiguous chunk of this CTA, contiguous sub-chunk of this thread (index order = rank order)
+  // contiguous chunk per CTA, contiguous segment of `rounds` 32-wide rounds per warp
   const int chunk = (n_cand + CLUSTER - 1) / CLUSTER;
   const int c_begin = min(n_cand, rank * chunk), c_end = min(n_cand, c_begin + chunk);
-  const int per_thread = (chunk + kSelThreads - 1) / kSelThreads;
-  const int t_begin = min(c_end, c_begin + tid * per_thread), t_end = min(c_end, t_begin + per_thread);
+  const int rounds = CACHED ? ITEMS : (chunk + kSelThreads - 1) / kSelThreads;
+  const int w_begin = c_begin + warp * rounds * 32;     // may lie beyond c_end (idle warp)
+
+  uint32_t key[R];
+  if (CACHED) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const int i = w_begin + r * 32 + lane;
+      key[r] = (i < c_end) ? order_key(__ldg(S + i)) : 0u;
+    }
+  }
 
   uint32_t prefix = 0;
   int k_rem = k_sel;
   if (k_sel > 0) {
+    for (int i = tid; i < kBins * 32; i += kSelThreads) sh.hist[i] = 0;
+    __syncthreads();
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
-      for (int i = tid; i < kBins * 32; i += kSelThreads) sh.hist[i] = 0;
-      __syncthreads();
-      for (int i = c_begin + tid; i < c_end; i += kSelThreads) {
-        const uint32_t u = order_key(S[i]);
-        const bool match = (pass == 0) || ((u ^ prefix) >> (shift + 8)) == 0;
-        if (match) atomicAdd(&sh.hist[((u >> shift) & 0xFFu) * 32 + lane], 1);
+      if (CACHED) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const uint32_t u = key[r];
+          const bool match = (w_begin + r * 32 + lane < c_end) &&
+                             ((pass == 0) || ((u ^ prefix) >> (shift + 8)) == 0);
+          if (match) atomicAdd(&sh.hist[((u >> shift) & 0xFFu) * 32 + lane], 1);
+        }
+      } else {
+#pragma unroll 4
+        for (int i = c_begin + tid; i < c_end; i += kSelThreads) {
+          const uint32_t u = order_key(__ldg(S + i));
+          const bool match = (pass == 0) || ((u ^ prefix) >> (shift + 8)) == 0;
+          if (match) atomicAdd(&sh.hist[((u >> shift) & 0xFFu) * 32 + lane], 1);
+        }
       }
       __syncthreads();
       {
-        // 4 threads per bin, each sums 8 lane counters
+        // 4 threads per bin, each sums (and clears for the next pass) 8 lane counters
         const int bin = tid >> 2, part = tid & 3;
         int s = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) s += sh.hist[bin * 32 + ((part * 8 + i + bin) & 31)];
+        for (int i = 0; i < 8; ++i) {
+          int* c = &sh.hist[bin * 32 + ((part * 8 + i + bin) & 31)];
+          s += *c;
+          *c = 0;
+        }
         s += __shfl_xor_sync(0xffffffffu, s, 1);
         s += __shfl_xor_sync(0xffffffffu, s, 2);
         if (part == 0) sh.block_hist[pass & 1][bin] = s;
       }
       cluster.sync();
-      if (warp == 0) {
-        // cluster-wide histogram, 8 bins per lane, highest bins first: lane 0 owns bins 255..248
-        int cnt[8], tot = 0;
+      if (tid < kBins) {               // one bin per thread: sum it over the cluster (DSMEM reads)
+        int c = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int bin = 255 - (lane * 8 + i);
-          int c = 0;
-          for (int r = 0; r < CLUSTER; ++r)
-            c += cluster.map_shared_rank(&sh.block_hist[pass & 1][0], r)[bin];
-          cnt[i] = c;
-          tot += c;
-        }
+        for (int r = 0; r < CLUSTER; ++r) c += cluster.map_shared_rank(&sh.block_hist[pass & 1][0], r)[tid];
+        sh.total_hist[tid] = c;
+      }
+      __syncthreads();
+      if (warp == 0) {
+        // 8 bins per lane, highest bins first: lane 0 owns bins 255..248
+        int cnt[8], tot = 0;
+        const int4 lo = *reinterpret_cast<const int4*>(&sh.total_hist[248 - lane * 8]);
+        const int4 hi = *reinterpret_cast<const int4*>(&sh.total_hist[252 - lane * 8]);
+        cnt[0] = hi.w; cnt[1] = hi.z; cnt[2] = hi.y; cnt[3] = hi.x;
+        cnt[4] = lo.w; cnt[5] = lo.z; cnt[6] = lo.y; cnt[7] = lo.x;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) tot += cnt[i];
         int incl = tot;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -128,91 +164,119 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
       __syncthreads();
       prefix |= static_cast<uint32_t>(sh.digit) << shift;
       k_rem = sh.k_rem;
-      __syncthreads();
     }
   }
   // prefix = image of the threshold score tau; k_rem = how many candidates equal to tau are kept
   const uint32_t tau = prefix;
   const int need_eq = (k_sel > 0) ? k_rem : 0;
 
-  // per-thread counts over its contiguous sub-chunk
+  // counting sweep: candidates above / equal to tau in this warp's segment (warp-uniform counts)
   int n_gt = 0, n_eq = 0;
   if (k_sel > 0) {
-    for (int i = t_begin; i < t_end; ++i) {
-      const uint32_t u = order_key(S[i]);
-      n_gt += (u > tau);
-      n_eq += (u == tau);
+#pragma unroll
+    for (int r = 0; r < (CACHED ? R : 1); ++r) {
+      for (int rr = (CACHED ? r : 0); rr < (CACHED ? r + 1 : rounds); ++rr) {
+        const int i = w_begin + rr * 32 + lane;
+        const uint32_t u = CACHED ? key[r] : ((i < c_end) ? order_key(__ldg(S + i)) : 0u);
+        n_gt += __popc(__ballot_sync(0xffffffffu, i < c_end && u > tau));
+        n_eq += __popc(__ballot_sync(0xffffffffu, i < c_end && u == tau));
+      }
     }
   }
-  // block-wide exclusive scans of both counts (packed: candidates per CTA < 2^31 / 2)
-  int gt_excl, eq_excl, gt_block, eq_block;
-  {
-    int gi = n_gt, ei = n_eq;
+  if (lane == 0) { sh.warp_tot[0][warp] = n_gt; sh.warp_tot[1][warp] = n_eq; }
+  __syncthreads();
+  if (warp == 0) {                   // exclusive scan over the 32 warps
+    int a = sh.warp_tot[0][lane], e = sh.warp_tot[1][lane];
+    const int a0 = a, e0 = e;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int a = __shfl_up_sync(0xffffffffu, gi, o), e = __shfl_up_sync(0xffffffffu, ei, o);
-      if (lane >= o) { gi += a; ei += e; }
+      const int va = __shfl_up_sync(0xffffffffu, a, o), ve = __shfl_up_sync(0xffffffffu, e, o);
+      if (lane >= o) { a += va; e += ve; }
     }
-    if (lane == 31) { sh.warp_tot[0][warp] = gi; sh.warp_tot[1][warp] = ei; }
-    __syncthreads();
-    if (warp == 0) {
-      int a = sh.warp_tot[0][lane], e = sh.warp_tot[1][lane];
-      const int a0 = a, e0 = e;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int va = __shfl_up_sync(0xffffffffu, a, o), ve = __shfl_up_sync(0xffffffffu, e, o);
-        if (lane >= o) { a += va; e += ve; }
-      }
-      sh.warp_tot[0][lane] = a - a0;
-      sh.warp_tot[1][lane] = e - e0;
-      if (lane == 31) { sh.counts[0] = a; sh.counts[1] = e; }
-    }
-    __syncthreads();
-    gt_excl = sh.warp_tot[0][warp] + gi - n_gt;
-    eq_excl = sh.warp_tot[1][warp] + ei - n_eq;
-    gt_block = sh.counts[0];
-    eq_block = sh.counts[1];
+    sh.warp_tot[0][lane] = a - a0;
+    sh.warp_tot[1][lane] = e - e0;
+    if (lane == 31) { sh.counts[0] = a; sh.counts[1] = e; }
   }
+  __syncthreads();
+  const int gt_excl = sh.warp_tot[0][warp], eq_excl = sh.warp_tot[1][warp];
   cluster.sync();
   // candidates kept by lower-ranked CTAs (they hold lower indices)
-  int eq_before = 0, kept_before = 0;
-  for (int r = 0; r < rank; ++r) {
-    const int* c = cluster.map_shared_rank(&sh.counts[0], r);
-    const int g_r = c[0], e_r = c[1];
-    kept_before += g_r + max(0, min(e_r, need_eq - eq_before));
-    eq_before += e_r;
+  int g_r[CLUSTER], e_r[CLUSTER];
+#pragma unroll
+  for (int r = 0; r < CLUSTER; ++r) {              // all remote reads in flight at once
+    const int2 c = *reinterpret_cast<const int2*>(cluster.map_shared_rank(&sh.counts[0], r));
+    g_r[r] = c.x;
+    e_r[r] = c.y;
   }
-  (void)gt_block; (void)eq_block;
+  int eq_before = 0, kept_before = 0;
+#pragma unroll
+  for (int r = 0; r < CLUSTER; ++r) {
+    if (r < rank) {
+      kept_before += g_r[r] + max(0, min(e_r[r], need_eq - eq_before));
+      eq_before += e_r[r];
+    }
+  }
   if (k_sel > 0) {
-    int eq_rank = eq_before + eq_excl;                       // rank of my first tau-valued candidate
-    const int eq_kept_before_me = min(eq_rank, need_eq) - min(eq_before, need_eq);
-    int pos = kept_before + gt_excl + eq_kept_before_me;
-    for (int i = t_begin; i < t_end; ++i) {
-      const uint32_t u = order_key(S[i]);
-      bool keep = u > tau;
-      if (u == tau) { keep = eq_rank < need_eq; ++eq_rank; }
-      if (keep) out[pos++] = i;
+    int eq_run = eq_before + eq_excl;                        // rank of the segment's first tau-valued candidate
+    int pos = kept_before + gt_excl + min(eq_run, need_eq) - min(eq_before, need_eq);
+#pragma unroll
+    for (int r = 0; r < (CACHED ? R : 1); ++r) {
+      for (int rr = (CACHED ? r : 0); rr < (CACHED ? r + 1 : rounds); ++rr) {
+        const int i = w_begin + rr * 32 + lane;
+        const uint32_t u = CACHED ? key[r] : ((i < c_end) ? order_key(__ldg(S + i)) : 0u);
+        const bool is_eq = i < c_end && u == tau;
+        const uint32_t be = __ballot_sync(0xffffffffu, is_eq);
+        const bool keep = i < c_end && (u > tau || (is_eq && eq_run + __popc(be & lt_mask) < need_eq));
+        const uint32_t bk = __ballot_sync(0xffffffffu, keep);
+        if (keep) out[pos + __popc(bk & lt_mask)] = i;
+        pos += __popc(bk);
+        eq_run += __popc(be);
+      }
     }
   }
   if (rank == 0 && tid < w) out[k_sel + tid] = n_cand + tid;   // the window, always kept
   cluster.sync();   // no CTA may exit while others still read its shared memory
 }
 
-cudaError_t launch_select(const SelectParams& p, int n_rows, int batch, cudaStream_t stream) {
-  constexpr int kCluster = 8;
+namespace {
+
+template <int CLUSTER, int ITEMS>
+cudaError_t launch_select_t(const SelectParams& p, int n_rows, int batch, cudaStream_t stream) {
+  if (CLUSTER > 8) {
+    static bool configured = false;
+    if (!configured) {
+      cudaError_t e = cudaFuncSetAttribute(select_topk_kernel<CLUSTER, ITEMS>,
+                                           cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+      if (e != cudaSuccess) return e;
+      configured = true;
+    }
+  }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(kCluster, n_rows, batch);
+  cfg.gridDim = dim3(CLUSTER, n_rows, batch);
   cfg.blockDim = dim3(kSelThreads);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = kCluster;
+  attr[0].val.clusterDim.x = CLUSTER;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, select_topk_kernel<kCluster>, p);
+  return cudaLaunchKernelEx(&cfg, select_topk_kernel<CLUSTER, ITEMS>, p);
+}
+
+}  // namespace
+
+cudaError_t launch_select(const SelectParams& p, int n_rows, int batch, int max_len, cudaStream_t stream) {
+  // 8-CTA clusters: every problem of a layer (KV heads plus the TSP row) is resident at once on a
+  // 148-SM part.  The per-thread register cache is picked from the longest sequence.
+  const long long per_cta = (static_cast<long long>(max_len) + 7) / 8;
+  if (per_cta <= 4 * kSelThreads) return launch_select_t<8, 4>(p, n_rows, batch, stream);
+  if (per_cta <= 8 * kSelThreads) return launch_select_t<8, 8>(p, n_rows, batch, stream);
+  if (per_cta <= 16 * kSelThreads) return launch_select_t<8, 16>(p, n_rows, batch, stream);
+  if (per_cta <= 32 * kSelThreads) return launch_select_t<8, 32>(p, n_rows, batch, stream);
+  return launch_select_t<8, 0>(p, n_rows, batch, stream);
 }
 
 }  // namespace fastkv

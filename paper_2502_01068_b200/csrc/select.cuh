@@ -19,6 +19,6 @@ struct SelectParams {
   WorkspaceHeader* hdr;
 };
 
-cudaError_t launch_select(const SelectParams& p, int n_rows, int batch, cudaStream_t stream);
+cudaError_t launch_select(const SelectParams& p, int n_rows, int batch, int max_len, cudaStream_t stream);
 
 }  // namespace fastkv
