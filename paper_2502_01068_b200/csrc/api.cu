@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "compact.cuh"
@@ -37,7 +38,13 @@ struct Layout {
   int npad, tiles_per_cta, max_ranges;
   long long ld_logits;
   size_t off_counters, off_final, off_partial, off_logits, bytes, zero_bytes;
+  // single-pass path (score_fused.cu): same header, its own carving of the rest
+  bool fused_shape_ok;        // the shape fits the tensor-memory-resident design on a full B200
+  int f_rows;                 // un-pooled rows written by pass 2 (KV heads or query heads)
+  size_t f_off_counters, f_off_flags, f_off_final, f_off_partial, f_off_a, f_zero_bytes, f_bytes;
 };
+
+constexpr int kFusedMaxCtas = 148;      // SMs of a B200: one persistent CTA each
 
 Layout make_layout(const fastkv_shape& s) {
   Layout l;
@@ -63,6 +70,26 @@ Layout make_layout(const fastkv_shape& s) {
   l.off_logits = off;
   off += round_up(sizeof(float) * static_cast<size_t>(s.n_kv_heads) * l.npad * l.ld_logits, 256);
   l.bytes = off;
+
+  const int phases = s.batch * s.n_kv_heads;
+  const bool per_head = s.agg_order == FASTKV_POOL_THEN_GROUP;
+  l.fused_shape_ok = max_tiles <= static_cast<long long>(kFusedMaxCtas) * fused_slots(l.npad) &&
+                     (!per_head || G == 1 || G == 2 || G == 4 || G == 8);
+  l.f_rows = per_head ? s.n_q_heads : s.n_kv_heads;
+  off = sizeof(WorkspaceHeader);
+  l.f_off_counters = off;
+  off += round_up(sizeof(int) * phases, 256);
+  l.f_off_flags = off;
+  off += round_up(sizeof(int) * phases, 256);
+  l.f_zero_bytes = off;
+  l.f_off_final = off;
+  off += round_up(sizeof(float2) * static_cast<size_t>(phases) * l.npad, 256);
+  l.f_off_partial = off;
+  off += round_up(sizeof(float2) * static_cast<size_t>(phases) * kFusedMaxCtas * l.npad, 256);
+  l.f_off_a = off;
+  off += round_up(sizeof(float) * static_cast<size_t>(l.f_rows) * l.ld_logits, 256);
+  l.f_bytes = off;
+  if (l.f_bytes > l.bytes) l.bytes = l.f_bytes;     // one size serves whichever path runs
   return l;
 }
 
@@ -165,6 +192,22 @@ int encode_bf16_3d(CUtensorMap* map, const void* base, int dim, int heads, long 
   return FASTKV_OK;
 }
 
+// Persistent CTAs the single-pass scoring kernel may use: one per SM, capped at the count the
+// workspace is carved for; 0 if the device cannot be queried or has no cooperative launch.
+int fused_grid() {
+  static int ctas = -1;
+  if (ctas < 0) {
+    int dev = 0, sms = 0, coop = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop)
+      ctas = 0;
+    else
+      ctas = sms < kFusedMaxCtas ? sms : kFusedMaxCtas;
+  }
+  return ctas;
+}
+
 int check_device() {
   static int ok = -1;
   if (ok < 0) {
@@ -222,22 +265,60 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
                            G, s.window)))
     return rc;
 
-  cudaError_t e = cudaMemsetAsync(ws, 0, lay.zero_bytes, stream);
+  const float scale = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / std::sqrt(static_cast<float>(s.head_dim));
+  const float scale_log2 = scale * 1.4426950408889634f;
+  WorkspaceHeader* hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+  const long long max_tiles = (static_cast<long long>(s.max_len) + 127) / 128;
+  const int ctas = fused_grid();
+  const char* force = std::getenv("FASTKV_SCORE_PATH");        // "buffered" forces the two-pass path
+  const bool fused = lay.fused_shape_ok && ctas > 0 && max_tiles <= static_cast<long long>(ctas) * fused_slots(lay.npad) &&
+                     !(force && std::strcmp(force, "buffered") == 0);
+  cudaError_t e;
+  if (fused) {
+    // ---- single pass over K: logits stay in tensor memory ----
+    e = cudaMemsetAsync(ws, 0, lay.f_zero_bytes, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace header)");
+    FusedParams fp;
+    fp.batch = s.batch; fp.total_len = s.total_len; fp.n_kv_heads = s.n_kv_heads; fp.group = G;
+    fp.window = s.window; fp.n_rows = G * s.window; fp.q_layout = s.q_layout;
+    fp.slots = fused_slots(lay.npad); fp.per_head = s.agg_order == FASTKV_POOL_THEN_GROUP;
+    fp.scale_log2 = scale_log2; fp.cu_seqlens = s.cu_seqlens;
+    fp.a_out = reinterpret_cast<float*>(ws + lay.f_off_a); fp.ld_a = lay.ld_logits;
+    fp.partial = reinterpret_cast<float2*>(ws + lay.f_off_partial);
+    fp.counters = reinterpret_cast<int*>(ws + lay.f_off_counters);
+    fp.hdr = hdr;
+    e = launch_score_fused(s.head_dim, lay.npad, tmap_k, tmap_q, fp, ctas, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "score_fused_kernel launch");
+    ++g_launches;
+    PoolRowsParams rp;
+    rp.total_len = s.total_len; rp.n_kv_heads = s.n_kv_heads; rp.group = G; rp.window = s.window;
+    rp.per_head = fp.per_head; rp.pool_kernel = s.pool_kernel; rp.pool_mode = s.pool_mode;
+    rp.cu_seqlens = s.cu_seqlens; rp.a = fp.a_out; rp.ld_a = lay.ld_logits;
+    rp.scores_kv = scores_kv; rp.ld_scores = s.total_len; rp.scores_tsp = scores_tsp;
+    if (sizeof(float) * static_cast<size_t>(lay.f_rows) * (kPoolKeys + s.pool_kernel) > 200 * 1024)
+      return fail(FASTKV_ERR_UNSUPPORTED, "heads x pool halo do not fit the pooling kernel's shared memory");
+    e = launch_pool_rows(rp, s.max_len, s.batch, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "pool_rows_kernel launch");
+    ++g_launches;
+    return FASTKV_OK;
+  }
+
+  // ---- two passes with buffered logits: any sequence length ----
+  e = cudaMemsetAsync(ws, 0, lay.zero_bytes, stream);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace header)");
 
   ScoreParams sp;
   sp.batch = s.batch; sp.total_len = s.total_len; sp.n_kv_heads = s.n_kv_heads; sp.group = G;
   sp.window = s.window; sp.n_rows = G * s.window; sp.q_layout = s.q_layout;
   sp.tiles_per_cta = lay.tiles_per_cta; sp.max_ranges = lay.max_ranges;
-  const float scale = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / std::sqrt(static_cast<float>(s.head_dim));
-  sp.scale_log2 = scale * 1.4426950408889634f;
-  sp.cu_seqlens = s.batch > 1 || s.cu_seqlens ? s.cu_seqlens : nullptr;
+  sp.scale_log2 = scale_log2;
+  sp.cu_seqlens = s.cu_seqlens;
   sp.logits = reinterpret_cast<float*>(ws + lay.off_logits);
   sp.ld_logits = lay.ld_logits;
   sp.partial = reinterpret_cast<float2*>(ws + lay.off_partial);
   sp.final_stats = reinterpret_cast<float2*>(ws + lay.off_final);
   sp.counters = reinterpret_cast<int*>(ws + lay.off_counters);
-  sp.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+  sp.hdr = hdr;
   dim3 grid(s.n_kv_heads, lay.max_ranges, s.batch);
   e = launch_score_logits(s.head_dim, lay.npad, tmap_k, tmap_q, sp, grid, stream);
   if (e != cudaSuccess) return cuda_fail(e, "score_logits_kernel launch");

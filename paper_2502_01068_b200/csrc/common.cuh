@@ -27,6 +27,13 @@ enum Site : int {
   SITE_SCORE_EPI_ACC_FULL = 4,
   SITE_SCORE_MMA_QFULL = 5,
   SITE_SCORE_SHORT_SEQUENCE = 6,
+  SITE_FUSED_EMPTY = 8,
+  SITE_FUSED_FULL = 9,
+  SITE_FUSED_Q_EMPTY = 10,
+  SITE_FUSED_Q_FULL = 11,
+  SITE_FUSED_ACC_FREE = 12,
+  SITE_FUSED_ACC_FULL = 13,
+  SITE_FUSED_FLAG = 14,
   SITE_COMPACT_INDEX = 16,
   SITE_SELECT_BUDGET = 17,
 };
@@ -197,6 +204,81 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// Online-softmax statistics (max m, sum l of exp2(x - m)) of two disjoint sets of logits combine as
+// m = max(m1, m2), l = l1 * 2^(m1 - m) + l2 * 2^(m2 - m); an empty set is (-inf, 0).
+__device__ __forceinline__ void merge_stats(float& m, float& l, float m2, float l2) {
+  if (m2 == -INFINITY) return;
+  const float mn = fmaxf(m, m2);
+  l = l * ex2(m - mn) + l2 * ex2(m2 - mn);     // m == -inf gives 2^-inf = 0 times l = 0
+  m = mn;
+}
+
+// Running softmax statistics of one thread over 32 query rows (one new logit per row).  t[x] must
+// hold s_x - m[x] with s_x = acc[x] * scale.  The running max may lag the true max by up to `slack`
+// (log2 units): in the common case no row needs rescaling anywhere in the warp and the update is
+// one exp2 per element, straight-line code with 32 independent dependency chains.
+constexpr float kLazyMaxSlackLog2 = 8.0f;
+
+template <int N>
+__device__ __forceinline__ void stats_update_unmasked(const float (&acc)[32], float* m, float* l, float scale,
+                                                      int n_valid) {
+  float t[32];
+  bool need = false;
+#pragma unroll
+  for (int x = 0; x < 32; ++x) {
+    t[x] = fmaf(acc[x], scale, -m[x]);
+    need |= (x < n_valid) && (t[x] > kLazyMaxSlackLog2);
+  }
+  if (__any_sync(0xffffffffu, need)) {             // some row's max moved: exact update, two exp2
+#pragma unroll
+    for (int x = 0; x < 32; ++x) {
+      if (x < n_valid) {
+        const float s = acc[x] * scale;
+        const float mn = fmaxf(m[x], s);
+        l[x] = l[x] * ex2(m[x] - mn) + ex2(s - mn);
+        m[x] = mn;
+      }
+    }
+  } else {
+#pragma unroll
+    for (int x = 0; x < 32; ++x)
+      if (x < n_valid) l[x] += ex2(t[x]);
+  }
+}
+
+// Same, for the tiles that overlap the observation window: row x sees the key only if visible[x].
+__device__ __forceinline__ void stats_update_masked(const float (&acc)[32], float* m, float* l, float scale,
+                                                    int n_valid, uint32_t visible) {
+#pragma unroll
+  for (int x = 0; x < 32; ++x) {
+    if (x < n_valid) {
+      const float s = ((visible >> x) & 1u) ? acc[x] * scale : -INFINITY;
+      const float mn = fmaxf(m[x], s);
+      const float ref = (mn == -INFINITY) ? 0.0f : mn;      // nothing seen yet: keep (m, l) = (-inf, 0)
+      l[x] = l[x] * ex2(m[x] - ref) + ex2(s - ref);
+      m[x] = mn;
+    }
+  }
+}
+
+// Merges `count` per-CTA statistics of row n (part[r * npad + n], r = first, first + stride, ...) in
+// a fixed order, with eight independent loads in flight at a time.
+__device__ __forceinline__ float2 merge_partials(const float2* part, int npad, int n, int first, int stride,
+                                                 int count) {
+  float m = -INFINITY, l = 0.0f;
+  for (int r0 = first; r0 < count; r0 += stride * 8) {
+    float2 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int r = r0 + j * stride;
+      v[j] = (r < count) ? __ldcg(&part[static_cast<size_t>(r) * npad + n]) : make_float2(-INFINITY, 0.0f);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) merge_stats(m, l, v[j].x, v[j].y);
+  }
+  return make_float2(m, l);
 }
 
 }  // namespace fastkv

@@ -22,7 +22,6 @@ constexpr int kTileKeys = 128;
 constexpr int kHalfBytes = kTileKeys * 128;   // one 64-column half of a K tile: 128 rows x 128 B
 constexpr int kEpilogueWarps = 4;
 constexpr int kScoreThreads = 32 * (2 + kEpilogueWarps);
-constexpr float kLazyMaxSlack = 8.0f;         // log2 units a row max may lag before rescaling
 
 template <int D, int NPAD>
 struct ScoreCfg {
@@ -176,32 +175,25 @@ score_logits_kernel(const __grid_constant__ CUtensorMap tmap_k,
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars->acc_empty[a]);
         }
+        const int n_valid = n_rows - c * 32;
+        float* const lg_c = lg + static_cast<size_t>(c * 32) * p.ld_logits + key;
         if (tile_unmasked) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int n = c * 32 + i;
-            if (n < n_rows) {
-              const float x = acc[i] * p.scale_log2;
-              lg[static_cast<size_t>(n) * p.ld_logits + key] = x;
-              if (x > m[n] + kLazyMaxSlack) { l[n] *= ex2(m[n] - x); m[n] = x; }
-              l[n] += ex2(x - m[n]);
-            }
-          }
+          for (int i = 0; i < 32; ++i)
+            if (i < n_valid) lg_c[static_cast<size_t>(i) * p.ld_logits] = acc[i] * p.scale_log2;
+          stats_update_unmasked<32>(acc, m + c * 32, l + c * 32, p.scale_log2, n_valid);
         } else if (key < L) {
+          uint32_t visible = 0;                          // causal: key i <= t_j, j = n / G
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int n = c * 32 + i;
-            if (n < n_rows) {
-              const int j = n / G;                       // window row of this query row
-              const bool visible = key <= win_start + j; // causal: key i <= t_j
-              const float x = visible ? acc[i] * p.scale_log2 : -INFINITY;
-              lg[static_cast<size_t>(n) * p.ld_logits + key] = x;
-              if (visible) {
-                if (x > m[n] + kLazyMaxSlack) { l[n] *= ex2(m[n] - x); m[n] = x; }
-                l[n] += ex2(x - m[n]);
-              }
-            }
-          }
+          for (int i = 0; i < 32; ++i)
+            if (i < n_valid && key <= win_start + (c * 32 + i) / G) visible |= 1u << i;
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (i < n_valid)
+              lg_c[static_cast<size_t>(i) * p.ld_logits] = ((visible >> i) & 1u) ? acc[i] * p.scale_log2 : -INFINITY;
+          stats_update_masked(acc, m + c * 32, l + c * 32, p.scale_log2, n_valid, visible);
+        } else {
+          stats_update_masked(acc, m + c * 32, l + c * 32, p.scale_log2, n_valid, 0u);   // warp-uniform call
         }
       }
     }
@@ -246,20 +238,26 @@ score_logits_kernel(const __grid_constant__ CUtensorMap tmap_k,
     is_last = (done == nranges - 1);
   }
   __syncthreads();
-  if (is_last && threadIdx.x < NPAD) {
-    __threadfence();
-    const int n = threadIdx.x;
-    float mm = -INFINITY;
-    for (int r = 0; r < nranges; ++r) mm = fmaxf(mm, __ldcg(&part[static_cast<size_t>(r) * NPAD + n]).x);
-    float ll = 0.0f;
-    for (int r = 0; r < nranges; ++r) {            // fixed order: the result does not depend on
-      const float2 s = __ldcg(&part[static_cast<size_t>(r) * NPAD + n]);   // which CTA came last
-      if (s.x != -INFINITY) ll += s.y * ex2(s.x - mm);
+  if (is_last) {
+    // 128 threads: row n = t % NPAD, CTAs r = t / NPAD, + 128 / NPAD, ...; the partitions are then
+    // combined in a fixed order, so the result does not depend on which CTA came last
+    __shared__ float2 merge_buf[128];
+    constexpr int kParts = 128 / NPAD;
+    const int t = threadIdx.x;
+    if (t < 128) {
+      __threadfence();
+      merge_buf[t] = merge_partials(part, NPAD, t % NPAD, t / NPAD, kParts, nranges);
     }
-    float2 out = make_float2(0.0f, 0.0f);
-    if (n < p.n_rows && ll > 0.0f && *abort_flag == 0) out = make_float2(mm, 1.0f / ll);
-    p.final_stats[(static_cast<size_t>(b) * p.n_kv_heads + g) * NPAD + n] = out;
-    if (n == 0) p.counters[b * p.n_kv_heads + g] = 0;
+    __syncthreads();
+    if (t < NPAD) {
+      float mm = -INFINITY, ll = 0.0f;
+#pragma unroll
+      for (int q = 0; q < kParts; ++q) merge_stats(mm, ll, merge_buf[q * NPAD + t].x, merge_buf[q * NPAD + t].y);
+      float2 out = make_float2(0.0f, 0.0f);
+      if (t < p.n_rows && ll > 0.0f && *abort_flag == 0) out = make_float2(mm, 1.0f / ll);
+      p.final_stats[(static_cast<size_t>(b) * p.n_kv_heads + g) * NPAD + t] = out;
+      if (t == 0) p.counters[b * p.n_kv_heads + g] = 0;
+    }
   }
 }
 

@@ -36,6 +36,38 @@ struct PoolParams {
   float* scores_tsp;          // [total_len] or null
 };
 
+// single-pass scoring (score_fused.cu): logits stay in tensor memory, nothing is buffered in HBM
+struct FusedParams {
+  int batch, total_len, n_kv_heads, group, window;
+  int n_rows;                 // G * w
+  int q_layout;
+  int slots;                  // accumulator slots in tensor memory = tiles a CTA may own per phase
+  int per_head;               // 1: write one un-pooled row per query head (POOL_THEN_GROUP)
+  float scale_log2;
+  const int* cu_seqlens;
+  float* a_out;               // [Hkv or Hq][ld_a] un-pooled scores
+  long long ld_a;
+  float2* partial;            // [phases][CTAs][NPAD]
+  int* counters;              // [phases] CTAs that published their statistics (zero before launch)
+  WorkspaceHeader* hdr;
+};
+
+struct PoolRowsParams {
+  int total_len, n_kv_heads, group, window, per_head;
+  int pool_kernel, pool_mode;
+  const int* cu_seqlens;
+  const float* a;
+  long long ld_a;
+  float* scores_kv;
+  long long ld_scores;
+  float* scores_tsp;
+};
+
+int fused_slots(int npad);
+cudaError_t launch_score_fused(int head_dim, int npad, const CUtensorMap& tmap_k, const CUtensorMap& tmap_q,
+                               const FusedParams& p, int grid, cudaStream_t stream);
+cudaError_t launch_pool_rows(const PoolRowsParams& p, int max_len, int batch, cudaStream_t stream);
+
 cudaError_t launch_score_logits(int head_dim, int npad, const CUtensorMap& tmap_k,
                                 const CUtensorMap& tmap_q, const ScoreParams& p, dim3 grid,
                                 cudaStream_t stream);

@@ -84,3 +84,34 @@ def test_llama8b_8k():
     o = oracle_layer(wl, x)
     st = check_layer(wl, x, g, o, what="8k")
     assert st["score_err"] < 2e-3
+
+
+def test_buffered_two_pass_path_still_matches(monkeypatch):
+    """Sequences too long for the tensor-memory-resident scoring kernel use the two-pass kernel with
+    buffered logits; FASTKV_SCORE_PATH=buffered selects it for any shape."""
+    monkeypatch.setenv("FASTKV_SCORE_PATH", "buffered")
+    for wl in (W.tiny(), small("buf", 600, [3000, 130, 1000], [300, 64, 200], [500, 20, 100])):
+        x = W.make_layer(wl)
+        for order in (B.GROUP_THEN_POOL, B.POOL_THEN_GROUP):
+            g = gpu_layer(wl, x, pool_mode=B.POOL_MAX, agg_order=order)
+            o = oracle_layer(wl, x, pool_mode=B.POOL_MAX, agg_order=order)
+            check_layer(wl, x, g, o, what="buffered")
+
+
+def test_sequence_longer_than_tensor_memory_capacity():
+    """L = 160 000 > 148 SMs x 8 tiles x 128 keys: falls back to the buffered path by itself."""
+    wl = small("long", 601, [160000], [4000], [8000], Hq=4, Hkv=1, d=64, hidden=64)
+    x = W.make_layer(wl)
+    g = gpu_layer(wl, x)
+    o = oracle_layer(wl, x)
+    check_layer(wl, x, g, o, what="160k")
+
+
+def test_group_sizes_and_wide_windows_on_the_fused_path():
+    for Hq, Hkv, w in [(8, 8, 8), (16, 8, 8), (16, 2, 8), (8, 2, 16), (4, 1, 16), (12, 4, 8)]:
+        wl = small("grp", 700 + Hq + Hkv + w, [2000], [300], [400], Hq=Hq, Hkv=Hkv, w=w)
+        x = W.make_layer(wl)
+        for order in (B.GROUP_THEN_POOL, B.POOL_THEN_GROUP):
+            g = gpu_layer(wl, x, agg_order=order, pool_mode=B.POOL_MAX)
+            o = oracle_layer(wl, x, agg_order=order, pool_mode=B.POOL_MAX)
+            check_layer(wl, x, g, o, what="G=%d w=%d order=%d" % (Hq // Hkv, w, order))
