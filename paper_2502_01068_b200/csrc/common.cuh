@@ -263,20 +263,53 @@ __device__ __forceinline__ void stats_update_masked(const float (&acc)[32], floa
   }
 }
 
+// The first logit of each row starts the statistics without any exp2: (m, l) = (s, 1).
+__device__ __forceinline__ void stats_init_unmasked(const float (&acc)[32], float* m, float* l, float scale,
+                                                    int n_valid) {
+#pragma unroll
+  for (int x = 0; x < 32; ++x) {
+    if (x < n_valid) {
+      m[x] = acc[x] * scale;
+      l[x] = 1.0f;
+    }
+  }
+}
+
+// Transposing butterfly over the 32 lanes of a warp: on entry every lane holds statistics (m[x], l[x])
+// of rows x = 0..31 for its own keys; on return lane r holds in (m[0], l[0]) the statistics of row r
+// merged over all 32 lanes.  31 exchanges of a pair instead of 32 x 5 shuffle reductions.
+__device__ __forceinline__ void stats_transpose_merge(float* m, float* l, int lane) {
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) {
+    const bool upper = (lane & o) != 0;
+#pragma unroll
+    for (int i = 0; i < o; ++i) {
+      // this lane keeps row i (lower) or i + o (upper) of the current 2*o rows and sends the other
+      const float send_m = upper ? m[i] : m[i + o], send_l = upper ? l[i] : l[i + o];
+      float keep_m = upper ? m[i + o] : m[i], keep_l = upper ? l[i + o] : l[i];
+      const float got_m = __shfl_xor_sync(0xffffffffu, send_m, o);
+      const float got_l = __shfl_xor_sync(0xffffffffu, send_l, o);
+      merge_stats(keep_m, keep_l, got_m, got_l);
+      m[i] = keep_m;
+      l[i] = keep_l;
+    }
+  }
+}
+
 // Merges `count` per-CTA statistics of row n (part[r * npad + n], r = first, first + stride, ...) in
-// a fixed order, with eight independent loads in flight at a time.
+// a fixed order, with sixteen independent loads in flight at a time.
 __device__ __forceinline__ float2 merge_partials(const float2* part, int npad, int n, int first, int stride,
                                                  int count) {
   float m = -INFINITY, l = 0.0f;
-  for (int r0 = first; r0 < count; r0 += stride * 8) {
-    float2 v[8];
+  for (int r0 = first; r0 < count; r0 += stride * 16) {
+    float2 v[16];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < 16; ++j) {
       const int r = r0 + j * stride;
       v[j] = (r < count) ? __ldcg(&part[static_cast<size_t>(r) * npad + n]) : make_float2(-INFINITY, 0.0f);
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) merge_stats(m, l, v[j].x, v[j].y);
+    for (int j = 0; j < 16; ++j) merge_stats(m, l, v[j].x, v[j].y);
   }
   return make_float2(m, l);
 }

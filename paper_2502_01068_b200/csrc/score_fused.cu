@@ -226,7 +226,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           tmem_ld_32x32(lane_base + slot * NPAD + c * 32, acc);
           const int n_valid = n_rows - c * 32;
           if (tile_unmasked) {
-            stats_update_unmasked<32>(acc, m + c * 32, l + c * 32, p.scale_log2, n_valid);
+            if (i == 0) stats_init_unmasked(acc, m + c * 32, l + c * 32, p.scale_log2, n_valid);
+            else stats_update_unmasked<32>(acc, m + c * 32, l + c * 32, p.scale_log2, n_valid);
           } else {
             uint32_t visible = 0;                        // causal: key i <= t_j, j = n / G
             if (key < w.L) {
@@ -239,16 +240,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         }
       }
       if (!ok) break;
-      // lanes -> warp: after the butterfly, lane r holds row r (and r + 32 when NPAD = 64)
+      // lanes -> warp: after the butterfly lane r holds row c * 32 + r in entry c * 32
 #pragma unroll
-      for (int n = 0; n < NPAD; ++n) {
-        float mm = m[n];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
-        float ll = (m[n] == -INFINITY) ? 0.0f : l[n] * ex2(m[n] - mm);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ll += __shfl_xor_sync(0xffffffffu, ll, o);
-        if (lane == (n & 31)) warp_stats[quarter * NPAD + n] = make_float2(mm, ll);
+      for (int c = 0; c < NPAD / 32; ++c) {
+        stats_transpose_merge(m + c * 32, l + c * 32, lane);
+        warp_stats[quarter * NPAD + c * 32 + lane] = make_float2(m[c * 32], l[c * 32]);
       }
       group_sync<1>();
       if (at < NPAD) {                                   // warps -> CTA, publish
@@ -256,10 +252,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
         for (int q = 0; q < kGroupWarps; ++q) merge_stats(mm, ll, warp_stats[q * NPAD + at].x, warp_stats[q * NPAD + at].y);
         p.partial[(static_cast<size_t>(phase) * ncta + cta) * NPAD + at] = make_float2(mm, ll);
-        __threadfence();
       }
       group_sync<1>();                                   // also: warp_stats may be rewritten next phase
-      if (at == 0) red_release_add(p.counters + phase, 1);
+      if (at == 0) red_release_add(p.counters + phase, 1);   // release: cumulative over the barrier
     }
   } else {
     // ---------------- group B: pass 2, normalise and sum over window rows / group, free the slots ----------------
