@@ -167,7 +167,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     // ---------------- MMA issuer: accumulators form a ring of kSlots tensor-memory slots ----------------
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16_f32(kTileKeys, NPAD);
-      int it = 0, u = 0;
+      int it = 0, u = 0, seq = 0;
       bool ok = true;
       for (int phase = 0; ok && phase < n_phases; ++phase) {
         const PhaseWork w = phase_work(p, phase, cta, ncta);
@@ -177,8 +177,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         if (!ok) break;
         const uint32_t q_addr = smem_u32(smem_q + h * Cfg::kQBytes);
         for (int i = 0; i < w.n; ++i, ++it) {
-          const int s = it % Cfg::kStages, slot = it % Cfg::kSlots;
-          ok = mbar_wait_bounded(&bars->acc_free[slot], ((it / Cfg::kSlots) & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_ACC_FREE) &&
+          const int s = it % Cfg::kStages, slot = (seq + i) % Cfg::kSlots, use = (seq + i) / Cfg::kSlots;
+          ok = mbar_wait_bounded(&bars->acc_free[slot], (use & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_ACC_FREE) &&
                mbar_wait_bounded(&bars->full[s], (it / Cfg::kStages) & 1, abort_flag, p.hdr, SITE_FUSED_FULL);
           if (!ok) break;
           tc_fence_after_sync();
@@ -193,28 +193,31 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           tc_commit(&bars->acc_full[slot]);
         }
         if (ok) tc_commit(&bars->q_empty[h]);
+        seq += w.n + 1;                                  // the phase's tiles plus its statistics slot
         ++u;
       }
     }
   } else if (warp < 2 + kGroupWarps) {
-    // ---------------- group A: pass 1, running (max, sum) per query row; publish per phase ----------------
+    // ---------------- group A: pass 1 ----------------
+    // Per tile: e = exp2(s - m) with a per-(lane, row) reference m, written back over the logits;
+    // l += e.  m is the row's first logit and moves only when a logit exceeds it by more than the
+    // slack (rare); then l and the e already stored for the phase's earlier tiles are rescaled,
+    // so that at the end of the phase every stored e of a lane is relative to its final m.
     const int quarter = warp & 3;
     const int key_in_tile = quarter * 32 + lane;
     const int at = threadIdx.x - 64;                    // 0..127 within the group
     const int n_rows = p.n_rows, G = p.group;
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-    int it = 0;
+    int seq = 0;
     bool ok = true;
     for (int phase = 0; ok && phase < n_phases; ++phase) {
       const PhaseWork w = phase_work(p, phase, cta, ncta);
       if (w.n == 0) continue;
       float m[NPAD], l[NPAD];
-#pragma unroll
-      for (int n = 0; n < NPAD; ++n) { m[n] = -INFINITY; l[n] = 0.0f; }
       const int win_start = w.L - p.window;
-      for (int i = 0; i < w.n; ++i, ++it) {
-        const int slot = it % Cfg::kSlots;
-        ok = mbar_wait_bounded(&bars->acc_full[slot], (it / Cfg::kSlots) & 1, abort_flag, p.hdr, SITE_FUSED_ACC_FULL);
+      for (int i = 0; i < w.n; ++i) {
+        const int slot = (seq + i) % Cfg::kSlots, use = (seq + i) / Cfg::kSlots;
+        ok = mbar_wait_bounded(&bars->acc_full[slot], use & 1, abort_flag, p.hdr, SITE_FUSED_ACC_FULL);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after_sync();
@@ -222,24 +225,77 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         const bool tile_unmasked = (w.t0 + i + 1) * kTileKeys <= win_start;
 #pragma unroll
         for (int c = 0; c < NPAD / 32; ++c) {
-          float acc[32];
-          tmem_ld_32x32(lane_base + slot * NPAD + c * 32, acc);
+          float e[32];
+          const uint32_t taddr = lane_base + slot * NPAD + c * 32;
+          tmem_ld_32x32(taddr, e);
           const int n_valid = n_rows - c * 32;
-          if (tile_unmasked) {
-            if (i == 0) stats_init_unmasked(acc, m + c * 32, l + c * 32, p.scale_log2, n_valid);
-            else stats_update_unmasked<32>(acc, m + c * 32, l + c * 32, p.scale_log2, n_valid);
-          } else {
-            uint32_t visible = 0;                        // causal: key i <= t_j, j = n / G
+          uint32_t visible = 0xffffffffu;                // causal: key i <= t_j, j = n / G
+          if (!tile_unmasked) {
+            visible = 0;
             if (key < w.L) {
 #pragma unroll
               for (int x = 0; x < 32; ++x)
                 if (x < n_valid && key <= win_start + (c * 32 + x) / G) visible |= 1u << x;
             }
-            stats_update_masked(acc, m + c * 32, l + c * 32, p.scale_log2, n_valid, visible);
           }
+          float* const mc = m + c * 32;
+          float* const lc = l + c * 32;
+          if (i == 0) {
+#pragma unroll
+            for (int x = 0; x < 32; ++x) {
+              const bool vis = (visible >> x) & 1u;
+              mc[x] = vis ? e[x] * p.scale_log2 : -INFINITY;
+              e[x] = vis ? 1.0f : 0.0f;
+              lc[x] = e[x];
+            }
+          } else {
+            bool need = false;                           // s - m is +inf while m = -inf
+#pragma unroll
+            for (int x = 0; x < 32; ++x)
+              need |= (x < n_valid) && ((visible >> x) & 1u) && (fmaf(e[x], p.scale_log2, -mc[x]) > kLazyMaxSlackLog2);
+            if (__any_sync(0xffffffffu, need)) {         // rare: some reference moves up to its new logit
+              float fac[32];
+#pragma unroll
+              for (int x = 0; x < 32; ++x) {
+                const float sx = e[x] * p.scale_log2;
+                const bool mv = (x < n_valid) && ((visible >> x) & 1u) && (sx - mc[x] > kLazyMaxSlackLog2);
+                fac[x] = (mv && mc[x] != -INFINITY) ? ex2(mc[x] - sx) : 1.0f;      // 2^(m_old - m_new)
+                mc[x] = mv ? sx : mc[x];
+                lc[x] *= fac[x];
+              }
+              for (int j = 0; j < i; ++j) {              // earlier tiles of the phase: e *= 2^(m_old - m_new)
+                const uint32_t tj = lane_base + ((seq + j) % Cfg::kSlots) * NPAD + c * 32;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  float old[8];
+                  tmem_ld_32x8(tj + q * 8, old);
+#pragma unroll
+                  for (int x = 0; x < 8; ++x) old[x] *= fac[q * 8 + x];
+                  tmem_st_32x8(tj + q * 8, old);
+                }
+              }
+            }
+#pragma unroll
+            for (int x = 0; x < 32; ++x) {
+              e[x] = ((visible >> x) & 1u) ? ex2(fmaf(e[x], p.scale_log2, -mc[x])) : 0.0f;
+              lc[x] += e[x];
+            }
+          }
+          tmem_st_32x32(taddr, e);
         }
       }
       if (!ok) break;
+      // the lane's final references go into the phase's statistics slot for group B
+      const int sslot = (seq + w.n) % Cfg::kSlots, suse = (seq + w.n) / Cfg::kSlots;
+      ok = mbar_wait_bounded(&bars->acc_free[sslot], (suse & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_ACC_FREE);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after_sync();
+#pragma unroll
+      for (int c = 0; c < NPAD / 32; ++c)
+        tmem_st_32x32(lane_base + sslot * NPAD + c * 32, *reinterpret_cast<const float(*)[32]>(m + c * 32));
+      tmem_wait_st();
+      tc_fence_before_sync();
       // lanes -> warp: after the butterfly lane r holds row c * 32 + r in entry c * 32
 #pragma unroll
       for (int c = 0; c < NPAD / 32; ++c) {
@@ -254,22 +310,27 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         p.partial[(static_cast<size_t>(phase) * ncta + cta) * NPAD + at] = make_float2(mm, ll);
       }
       group_sync<1>();                                   // also: warp_stats may be rewritten next phase
-      if (at == 0) red_release_add(p.counters + phase, 1);   // release: cumulative over the barrier
+      if (at == 0) {
+        red_release_add(p.counters + phase, 1);          // release: cumulative over the barrier
+        mbar_arrive(&bars->acc_full[sslot]);             // keeps this slot's full/free parities in step
+      }
+      seq += w.n + 1;
     }
   } else {
-    // ---------------- group B: pass 2, normalise and sum over window rows / group, free the slots ----------------
+    // ---------------- group B: pass 2 ----------------
+    // Once every CTA of the phase has published: merge the statistics into (M_r, 1 / l_r), turn the
+    // lane's references into factors f = 2^(m - M_r) / l_r, and sum e * f over the window rows (and
+    // the group) of each key.  No exponential per logit here.
     const int quarter = warp & 3;
     const int key_in_tile = quarter * 32 + lane;
     const int bt = threadIdx.x - 64 - kGroupWarps * 32;   // 0..127 within the group
     const int n_rows = p.n_rows, G = p.group;
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
     constexpr int kParts = kGroupWarps * 32 / NPAD;
-    int it = 0;
-    bool ok = true;
-    for (int phase = 0; ok && phase < n_phases; ++phase) {
+    int seq = 0;
+    for (int phase = 0; phase < n_phases; ++phase) {
       const PhaseWork w = phase_work(p, phase, cta, ncta);
       if (w.n == 0) continue;
-      // every CTA that owns tiles of this phase has published its statistics?
       if (bt == 0) {
         const int* ctr = p.counters + phase;
         if (ld_acquire(ctr) < w.nact) {
@@ -297,18 +358,25 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         norm[bt] = (bt < n_rows && ll > 0.0f) ? make_float2(mm, 1.0f / ll) : make_float2(0.0f, 0.0f);
       }
       group_sync<2>();
-      float nm[NPAD], nil[NPAD];                         // -(row max) and 1 / (row sum)
+      tc_fence_after_sync();
+      const int sslot = (seq + w.n) % Cfg::kSlots;
+      float f[NPAD];
 #pragma unroll
-      for (int n = 0; n < NPAD; ++n) { const float2 st = norm[n]; nm[n] = -st.x; nil[n] = st.y; }
-      const int win_start = w.L - p.window;
-      for (int i = 0; i < w.n; ++i, ++it) {
-        const int slot = it % Cfg::kSlots;
-        ok = mbar_wait_bounded(&bars->acc_full[slot], (it / Cfg::kSlots) & 1, abort_flag, p.hdr, SITE_FUSED_ACC_FULL);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        tc_fence_after_sync();
+      for (int c = 0; c < NPAD / 32; ++c) {
+        float mref[32];
+        tmem_ld_32x32(lane_base + sslot * NPAD + c * 32, mref);
+#pragma unroll
+        for (int x = 0; x < 32; ++x) {
+          const float2 st = norm[c * 32 + x];
+          f[c * 32 + x] = (c * 32 + x < n_rows) ? ex2(mref[x] - st.x) * st.y : 0.0f;   // m = -inf gives 0
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->acc_free[sslot]);
+      for (int i = 0; i < w.n; ++i) {
+        const int slot = (seq + i) % Cfg::kSlots;
         const int key = (w.t0 + i) * kTileKeys + key_in_tile;
-        const bool tile_unmasked = (w.t0 + i + 1) * kTileKeys <= win_start;
         float a_g = 0.0f;
         float a_h[8];                                    // per query head of the group (G in {1,2,4,8})
 #pragma unroll
@@ -324,13 +392,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           }
           const int n_valid = n_rows - c * 32;
 #pragma unroll
-          for (int x = 0; x < 32; ++x)
-            pr[x] = (x < n_valid) ? ex2(fmaf(pr[x], p.scale_log2, nm[c * 32 + x])) * nil[c * 32 + x] : 0.0f;
-          if (!tile_unmasked) {                          // causal: key i <= t_j, j = n / G
-#pragma unroll
-            for (int x = 0; x < 32; ++x)
-              if (x < n_valid && key > win_start + (c * 32 + x) / G) pr[x] = 0.0f;
-          }
+          for (int x = 0; x < 32; ++x) pr[x] = (x < n_valid) ? pr[x] * f[c * 32 + x] : 0.0f;
           if (!p.per_head) {
 #pragma unroll
             for (int x = 0; x < 32; x += 4) a_g += (pr[x] + pr[x + 1]) + (pr[x + 2] + pr[x + 3]);
@@ -354,6 +416,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         }
       }
       group_sync<2>();                                   // norm / merge_buf are rewritten next phase
+      seq += w.n + 1;
     }
   }
 
@@ -414,7 +477,7 @@ __global__ void __launch_bounds__(kPoolThreads) pool_rows_kernel(const PoolRowsP
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
-int fused_slots(int npad) { return 512 / npad; }
+int fused_slots(int npad) { return 512 / npad - 1; }   // one slot per phase carries the lanes' references
 
 template <int D, int NPAD>
 static cudaError_t launch_fused_t(const CUtensorMap& tk, const CUtensorMap& tq, const FusedParams& p, int grid,

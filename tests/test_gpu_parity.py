@@ -115,3 +115,26 @@ def test_group_sizes_and_wide_windows_on_the_fused_path():
             g = gpu_layer(wl, x, agg_order=order, pool_mode=B.POOL_MAX)
             o = oracle_layer(wl, x, agg_order=order, pool_mode=B.POOL_MAX)
             check_layer(wl, x, g, o, what="G=%d w=%d order=%d" % (Hq // Hkv, w, order))
+
+
+@pytest.mark.parametrize("scale", [0.5, 2.0])
+def test_wide_logit_range_exercises_reference_rescaling(scale):
+    """With a large softmax scale the logits span far more than the slack the kernel allows between a
+    lane's reference and its running maximum, so stored exponentials get rescaled mid-phase.  Scores
+    only (most of them underflow to zero on both sides, which makes the selection a tie lottery)."""
+    import oracle
+    from tests.parity import SCORE_RTOL, dev
+    for L, Hq, Hkv, d, w in [(5000, 8, 2, 128, 8), (1500, 4, 1, 64, 8), (20000, 8, 2, 128, 16)]:
+        wl = small("wide", 800 + L, [L], [w], [w], Hq=Hq, Hkv=Hkv, d=d, w=w)
+        x = W.make_layer(wl, with_v=False, with_hidden=False)
+        shape = B.make_shape(total_len=L, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, window=w, softmax_scale=scale)
+        ws = torch.empty(B.fastkv_workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+        s_kv = torch.empty((Hkv, L), dtype=torch.float32, device="cuda")
+        s_tsp = torch.empty((L,), dtype=torch.float32, device="cuda")
+        B.fastkv_score(shape, dev(x.q_win), dev(x.k), s_kv, s_tsp, ws)
+        assert B.fastkv_device_status(ws)[0] == 0
+        ref_kv, ref_tsp, _ = oracle.scores(x.q_win, L - w, x.k, w, 7, scale=scale)
+        got = s_kv.cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - ref_kv) <= SCORE_RTOL * np.abs(ref_kv) + 1e-12)
+        np.testing.assert_allclose(got.sum(axis=1), ref_kv.sum(axis=1), rtol=1e-5)
+        assert np.all(np.abs(s_tsp.cpu().numpy() - ref_tsp) <= SCORE_RTOL * np.abs(ref_tsp) + 1e-12)
