@@ -73,8 +73,7 @@ Layout make_layout(const fastkv_shape& s) {
 
   const int phases = s.batch * s.n_kv_heads;
   const bool per_head = s.agg_order == FASTKV_POOL_THEN_GROUP;
-  l.fused_shape_ok = max_tiles <= static_cast<long long>(kFusedMaxCtas) * fused_slots(l.npad) &&
-                     (!per_head || G == 1 || G == 2 || G == 4 || G == 8);
+  l.fused_shape_ok = !per_head || G == 1 || G == 2 || G == 4 || G == 8;
   l.f_rows = per_head ? s.n_q_heads : s.n_kv_heads;
   off = sizeof(WorkspaceHeader);
   l.f_off_counters = off;
@@ -87,7 +86,7 @@ Layout make_layout(const fastkv_shape& s) {
   l.f_off_partial = off;
   off += round_up(sizeof(float2) * static_cast<size_t>(phases) * kFusedMaxCtas * l.npad, 256);
   l.f_off_a = off;
-  off += round_up(sizeof(float) * static_cast<size_t>(l.f_rows) * l.ld_logits, 256);
+  off += 2 * round_up(sizeof(float) * static_cast<size_t>(l.f_rows) * l.ld_logits, 256);   // two planes
   l.f_bytes = off;
   if (l.f_bytes > l.bytes) l.bytes = l.f_bytes;     // one size serves whichever path runs
   return l;
@@ -268,22 +267,24 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
   const float scale = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / std::sqrt(static_cast<float>(s.head_dim));
   const float scale_log2 = scale * 1.4426950408889634f;
   WorkspaceHeader* hdr = reinterpret_cast<WorkspaceHeader*>(ws);
-  const long long max_tiles = (static_cast<long long>(s.max_len) + 127) / 128;
   const int ctas = fused_grid();
   const char* force = std::getenv("FASTKV_SCORE_PATH");        // "buffered" forces the two-pass path
-  const bool fused = lay.fused_shape_ok && ctas > 0 && max_tiles <= static_cast<long long>(ctas) * fused_slots(lay.npad) &&
-                     !(force && std::strcmp(force, "buffered") == 0);
+  const bool fused = lay.fused_shape_ok && ctas > 0 && !(force && std::strcmp(force, "buffered") == 0);
   cudaError_t e;
   if (fused) {
-    // ---- single pass over K: logits stay in tensor memory ----
+    // ---- one HBM pass over K: persistent two-pipeline kernel ----
     e = cudaMemsetAsync(ws, 0, lay.f_zero_bytes, stream);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace header)");
     FusedParams fp;
     fp.batch = s.batch; fp.total_len = s.total_len; fp.n_kv_heads = s.n_kv_heads; fp.group = G;
     fp.window = s.window; fp.n_rows = G * s.window; fp.q_layout = s.q_layout;
-    fp.slots = fused_slots(lay.npad); fp.per_head = s.agg_order == FASTKV_POOL_THEN_GROUP;
+    fp.per_head = s.agg_order == FASTKV_POOL_THEN_GROUP;
     fp.scale_log2 = scale_log2; fp.cu_seqlens = s.cu_seqlens;
     fp.a_out = reinterpret_cast<float*>(ws + lay.f_off_a); fp.ld_a = lay.ld_logits;
+    fp.plane_stride = static_cast<long long>(round_up(sizeof(float) * static_cast<size_t>(lay.f_rows) * lay.ld_logits, 256) / sizeof(float));
+    const char* lead = std::getenv("FASTKV_FUSED_LEAD");     // tuning knob: phases of K kept in flight in L2
+    fp.max_lead = lead ? std::atoi(lead) : 3;
+    if (fp.max_lead < 1) fp.max_lead = 1;
     fp.partial = reinterpret_cast<float2*>(ws + lay.f_off_partial);
     fp.counters = reinterpret_cast<int*>(ws + lay.f_off_counters);
     fp.hdr = hdr;
@@ -293,7 +294,7 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
     PoolRowsParams rp;
     rp.total_len = s.total_len; rp.n_kv_heads = s.n_kv_heads; rp.group = G; rp.window = s.window;
     rp.per_head = fp.per_head; rp.pool_kernel = s.pool_kernel; rp.pool_mode = s.pool_mode;
-    rp.cu_seqlens = s.cu_seqlens; rp.a = fp.a_out; rp.ld_a = lay.ld_logits;
+    rp.cu_seqlens = s.cu_seqlens; rp.a = fp.a_out; rp.ld_a = lay.ld_logits; rp.plane_stride = fp.plane_stride;
     rp.scores_kv = scores_kv; rp.ld_scores = s.total_len; rp.scores_tsp = scores_tsp;
     if (sizeof(float) * static_cast<size_t>(lay.f_rows) * (kPoolKeys + s.pool_kernel) > 200 * 1024)
       return fail(FASTKV_ERR_UNSUPPORTED, "heads x pool halo do not fit the pooling kernel's shared memory");
@@ -303,7 +304,7 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
     return FASTKV_OK;
   }
 
-  // ---- two passes with buffered logits: any sequence length ----
+  // ---- two kernels with buffered logits: devices without cooperative launch, or on request ----
   e = cudaMemsetAsync(ws, 0, lay.zero_bytes, stream);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace header)");
 

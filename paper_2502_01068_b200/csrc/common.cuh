@@ -34,6 +34,8 @@ enum Site : int {
   SITE_FUSED_ACC_FREE = 12,
   SITE_FUSED_ACC_FULL = 13,
   SITE_FUSED_FLAG = 14,
+  SITE_FUSED_P1_DONE = 15,
+  SITE_FUSED_P2_DONE = 18,
   SITE_COMPACT_INDEX = 16,
   SITE_SELECT_BUDGET = 17,
 };
@@ -219,6 +221,21 @@ __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const float (&v)[3
         "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
       : "memory");
 }
+// 32 lanes x 16 consecutive fp32 columns -> 16 registers per thread
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
 // 8-column variants (used where registers are scarce)
 __device__ __forceinline__ void tmem_ld_32x8(uint32_t taddr, float (&v)[8]) {
   uint32_t r[8];
@@ -257,25 +274,21 @@ __device__ __forceinline__ void merge_stats(float& m, float& l, float m2, float 
   m = mn;
 }
 
-// Running softmax statistics of one thread over 32 query rows (one new logit per row).  t[x] must
-// hold s_x - m[x] with s_x = acc[x] * scale.  The running max may lag the true max by up to `slack`
-// (log2 units): in the common case no row needs rescaling anywhere in the warp and the update is
-// one exp2 per element, straight-line code with 32 independent dependency chains.
-constexpr float kLazyMaxSlackLog2 = 16.0f;
+// Running softmax statistics of one thread over N query rows (one new logit per row):
+// s_x = acc[x] * scale.  The running max may lag the true max by up to kLazyMaxSlackLog2 (log2
+// units): in the common case no row needs rescaling anywhere in the warp and the update is one
+// exp2 per element, straight-line code with N independent dependency chains.
+constexpr float kLazyMaxSlackLog2 = 8.0f;
 
 template <int N>
-__device__ __forceinline__ void stats_update_unmasked(const float (&acc)[32], float* m, float* l, float scale,
+__device__ __forceinline__ void stats_update_unmasked(const float (&acc)[N], float* m, float* l, float scale,
                                                       int n_valid) {
-  float t[32];
   bool need = false;
 #pragma unroll
-  for (int x = 0; x < 32; ++x) {
-    t[x] = fmaf(acc[x], scale, -m[x]);
-    need |= (x < n_valid) && (t[x] > kLazyMaxSlackLog2);
-  }
+  for (int x = 0; x < N; ++x) need |= (x < n_valid) && (fmaf(acc[x], scale, -m[x]) > kLazyMaxSlackLog2);
   if (__any_sync(0xffffffffu, need)) {             // some row's max moved: exact update, two exp2
 #pragma unroll
-    for (int x = 0; x < 32; ++x) {
+    for (int x = 0; x < N; ++x) {
       if (x < n_valid) {
         const float s = acc[x] * scale;
         const float mn = fmaxf(m[x], s);
@@ -285,16 +298,17 @@ __device__ __forceinline__ void stats_update_unmasked(const float (&acc)[32], fl
     }
   } else {
 #pragma unroll
-    for (int x = 0; x < 32; ++x)
-      if (x < n_valid) l[x] += ex2(t[x]);
+    for (int x = 0; x < N; ++x)
+      if (x < n_valid) l[x] += ex2(fmaf(acc[x], scale, -m[x]));
   }
 }
 
 // Same, for the tiles that overlap the observation window: row x sees the key only if visible[x].
-__device__ __forceinline__ void stats_update_masked(const float (&acc)[32], float* m, float* l, float scale,
+template <int N>
+__device__ __forceinline__ void stats_update_masked(const float (&acc)[N], float* m, float* l, float scale,
                                                     int n_valid, uint32_t visible) {
 #pragma unroll
-  for (int x = 0; x < 32; ++x) {
+  for (int x = 0; x < N; ++x) {
     if (x < n_valid) {
       const float s = ((visible >> x) & 1u) ? acc[x] * scale : -INFINITY;
       const float mn = fmaxf(m[x], s);
@@ -306,10 +320,11 @@ __device__ __forceinline__ void stats_update_masked(const float (&acc)[32], floa
 }
 
 // The first logit of each row starts the statistics without any exp2: (m, l) = (s, 1).
-__device__ __forceinline__ void stats_init_unmasked(const float (&acc)[32], float* m, float* l, float scale,
+template <int N>
+__device__ __forceinline__ void stats_init_unmasked(const float (&acc)[N], float* m, float* l, float scale,
                                                     int n_valid) {
 #pragma unroll
-  for (int x = 0; x < 32; ++x) {
+  for (int x = 0; x < N; ++x) {
     if (x < n_valid) {
       m[x] = acc[x] * scale;
       l[x] = 1.0f;
@@ -318,11 +333,13 @@ __device__ __forceinline__ void stats_init_unmasked(const float (&acc)[32], floa
 }
 
 // Transposing butterfly over the 32 lanes of a warp: on entry every lane holds statistics (m[x], l[x])
-// of rows x = 0..31 for its own keys; on return lane r holds in (m[0], l[0]) the statistics of row r
-// merged over all 32 lanes.  31 exchanges of a pair instead of 32 x 5 shuffle reductions.
+// of rows x = 0..N-1 (N = 16 or 32) for its own keys; on return lane r holds in (m[0], l[0]) the
+// statistics of row r % N merged over all 32 lanes.  N - 1 (+1) exchanges of a pair instead of
+// N x 5 shuffle reductions.
+template <int N>
 __device__ __forceinline__ void stats_transpose_merge(float* m, float* l, int lane) {
 #pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) {
+  for (int o = N / 2; o >= 1; o >>= 1) {
     const bool upper = (lane & o) != 0;
 #pragma unroll
     for (int i = 0; i < o; ++i) {
@@ -336,22 +353,31 @@ __device__ __forceinline__ void stats_transpose_merge(float* m, float* l, int la
       l[i] = keep_l;
     }
   }
+  if (N == 16) {                                   // lanes r and r + 16 hold the two halves of row r
+    const float got_m = __shfl_xor_sync(0xffffffffu, m[0], 16);
+    const float got_l = __shfl_xor_sync(0xffffffffu, l[0], 16);
+    float a_m = (lane & 16) ? got_m : m[0], a_l = (lane & 16) ? got_l : l[0];      // lower lane's half first:
+    const float b_m = (lane & 16) ? m[0] : got_m, b_l = (lane & 16) ? l[0] : got_l;  // same order on both lanes
+    merge_stats(a_m, a_l, b_m, b_l);
+    m[0] = a_m;
+    l[0] = a_l;
+  }
 }
 
 // Merges `count` per-CTA statistics of row n (part[r * npad + n], r = first, first + stride, ...) in
-// a fixed order, with sixteen independent loads in flight at a time.
+// a fixed order, with twenty independent loads in flight at a time.
 __device__ __forceinline__ float2 merge_partials(const float2* part, int npad, int n, int first, int stride,
                                                  int count) {
   float m = -INFINITY, l = 0.0f;
-  for (int r0 = first; r0 < count; r0 += stride * 16) {
-    float2 v[16];
+  for (int r0 = first; r0 < count; r0 += stride * 20) {
+    float2 v[20];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
+    for (int j = 0; j < 20; ++j) {
       const int r = r0 + j * stride;
       v[j] = (r < count) ? __ldcg(&part[static_cast<size_t>(r) * npad + n]) : make_float2(-INFINITY, 0.0f);
     }
 #pragma unroll
-    for (int j = 0; j < 16; ++j) merge_stats(m, l, v[j].x, v[j].y);
+    for (int j = 0; j < 20; ++j) merge_stats(m, l, v[j].x, v[j].y);
   }
   return make_float2(m, l);
 }

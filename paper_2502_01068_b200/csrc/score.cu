@@ -191,22 +191,17 @@ score_logits_kernel(const __grid_constant__ CUtensorMap tmap_k,
           for (int i = 0; i < 32; ++i)
             if (i < n_valid)
               lg_c[static_cast<size_t>(i) * p.ld_logits] = ((visible >> i) & 1u) ? acc[i] * p.scale_log2 : -INFINITY;
-          stats_update_masked(acc, m + c * 32, l + c * 32, p.scale_log2, n_valid, visible);
+          stats_update_masked<32>(acc, m + c * 32, l + c * 32, p.scale_log2, n_valid, visible);
         } else {
-          stats_update_masked(acc, m + c * 32, l + c * 32, p.scale_log2, n_valid, 0u);   // warp-uniform call
+          stats_update_masked<32>(acc, m + c * 32, l + c * 32, p.scale_log2, n_valid, 0u);   // warp-uniform call
         }
       }
     }
     // merge the 32 lanes of this warp: lane r ends up with row r (and r + 32) of the warp's stats
 #pragma unroll
-    for (int n = 0; n < NPAD; ++n) {
-      float mm = m[n];
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
-      float ll = (m[n] == -INFINITY) ? 0.0f : l[n] * ex2(m[n] - mm);
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) ll += __shfl_xor_sync(0xffffffffu, ll, o);
-      if (lane == (n & 31)) warp_stats[quarter * NPAD + n] = make_float2(mm, ll);
+    for (int c = 0; c < NPAD / 32; ++c) {
+      stats_transpose_merge<32>(m + c * 32, l + c * 32, lane);
+      warp_stats[quarter * NPAD + c * 32 + lane] = make_float2(m[c * 32], l[c * 32]);
     }
   }
 

@@ -36,17 +36,18 @@ struct PoolParams {
   float* scores_tsp;          // [total_len] or null
 };
 
-// single-pass scoring (score_fused.cu): logits stay in tensor memory, nothing is buffered in HBM
+// scoring with one HBM pass over K (score_fused.cu): nothing but the per-key sums is written to memory
 struct FusedParams {
   int batch, total_len, n_kv_heads, group, window;
   int n_rows;                 // G * w
   int q_layout;
-  int slots;                  // accumulator slots in tensor memory = tiles a CTA may own per phase
   int per_head;               // 1: write one un-pooled row per query head (POOL_THEN_GROUP)
   float scale_log2;
   const int* cu_seqlens;
-  float* a_out;               // [Hkv or Hq][ld_a] un-pooled scores
+  int max_lead;               // phases the HBM pipeline may run ahead of the re-read pipeline
+  float* a_out;               // [2][Hkv or Hq][ld_a] un-pooled scores, one plane per accumulator-column half
   long long ld_a;
+  long long plane_stride;     // elements between the two planes
   float2* partial;            // [phases][CTAs][NPAD]
   int* counters;              // [phases] CTAs that published their statistics (zero before launch)
   WorkspaceHeader* hdr;
@@ -56,14 +57,14 @@ struct PoolRowsParams {
   int total_len, n_kv_heads, group, window, per_head;
   int pool_kernel, pool_mode;
   const int* cu_seqlens;
-  const float* a;
+  const float* a;             // two planes, plane_stride apart; their sum is the un-pooled score
   long long ld_a;
+  long long plane_stride;
   float* scores_kv;
   long long ld_scores;
   float* scores_tsp;
 };
 
-int fused_slots(int npad);
 cudaError_t launch_score_fused(int head_dim, int npad, const CUtensorMap& tmap_k, const CUtensorMap& tmap_q,
                                const FusedParams& p, int grid, cudaStream_t stream);
 cudaError_t launch_pool_rows(const PoolRowsParams& p, int max_len, int batch, cudaStream_t stream);

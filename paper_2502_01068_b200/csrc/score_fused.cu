@@ -1,22 +1,24 @@
-// Window-query saliency scoring, single pass over K (Eq. 1 inner term; Sec. 4.2).
+// Window-query saliency scoring with one HBM pass over K (Eq. 1 inner term; Sec. 4.2).
 //
 // One persistent CTA per SM (cooperative launch, so all CTAs are resident).  The work is cut into
 // phases, one per (sequence, KV head); in a phase every CTA owns a run of consecutive 128-key
-// tiles.  The logits of a CTA's tiles stay in tensor memory between the two things that need them:
+// tiles.  Two tile pipelines run side by side in every CTA, each with its own TMA ring, its own
+// tcgen05 MMA issuer and its own ring of tensor-memory accumulators:
 //
-//   pass 1  (warp group A) running (max, sum of exp2) per query row over the CTA's tiles; the
-//           CTAs' statistics meet in global memory, counted by one counter per phase;
-//   pass 2  (warp group B) once every CTA of the phase has published, merge the statistics into
-//           the softmax normaliser (fixed order: identical in every CTA), then
-//           p = exp2(s - M_r) / l_r summed over the window rows (and the GQA group) of each key,
-//           read again from tensor memory -- K is streamed from HBM exactly once and no logit is
-//           ever written to memory.
+//   pipeline 1  streams the CTA's K tiles from HBM, forms the logits S^T = K_tile . Q_g^T and keeps
+//               a running (max, sum of exp2) per query row (warp group A); the CTAs' statistics of
+//               a phase meet in global memory, counted by one counter per phase;
+//   pipeline 2  follows one or two phases behind: once every CTA of the phase has published, it
+//               merges the statistics into the softmax normaliser (fixed order: identical in every
+//               CTA), loads the same K tiles again -- they are still in L2 -- recomputes the logits
+//               on the idle tensor cores and sums p = exp2(s - M_r) / l_r over the window rows
+//               (and the GQA group) of each key (warp group B).
 //
-// Tensor memory (512 columns) is a ring of accumulator slots: the MMA warp fills a slot, group A
-// reads it, group B reads it again and hands it back.  All tiles a CTA owns in one phase must be
-// in the ring at once (up to 16 tiles of 32 query rows), and the next phase's MMAs start as soon
-// as group B frees slots, so the TMA stream of K runs ahead of both passes.  Every wait (mbarrier
-// or counter) is bounded and ends in a status word instead of a hang.
+// Nothing but the final per-key sums is written to memory, HBM sees K once, and neither pipeline
+// holds anything across the grid-wide dependency except L2 lines, so the HBM stream of pipeline 1
+// never waits for other CTAs.  Pipeline 1 is throttled to stay at most kMaxLead phases ahead of
+// pipeline 2 so that the re-read really hits L2.  Every wait (mbarrier, counter, flag) is bounded
+// and ends in a status word instead of a hang.
 #include "score.cuh"
 
 namespace fastkv {
@@ -25,36 +27,39 @@ namespace {
 
 constexpr int kTileKeys = 128;
 constexpr int kHalfBytes = kTileKeys * 128;
-constexpr int kGroupWarps = 4;                 // warps per epilogue group (one per tensor-memory lane quarter)
-constexpr int kFusedThreads = 32 * (2 + 2 * kGroupWarps);
+constexpr int kGroupWarps = 8;                 // warps per epilogue group: 4 lane quarters x 2 column halves
+constexpr int kCtrlWarps = 4;                  // TMA 1, MMA 1, TMA 2, MMA 2
+constexpr int kFusedThreads = 32 * (kCtrlWarps + 2 * kGroupWarps);
+constexpr int kAcc = 4;                        // accumulators per pipeline
 
 template <int D, int NPAD>
 struct FusedCfg {
   static constexpr int KH = D / 64;
   static constexpr int kStageBytes = KH * kHalfBytes;
   static constexpr int kQBytes = KH * NPAD * 128;
-  static constexpr int kStages = (D == 128) ? (NPAD == 32 ? 6 : 5) : 8;
-  static constexpr int kSlots = 512 / NPAD;              // accumulators in tensor memory (a ring)
-  static constexpr int kTmemCols = 512;
+  static constexpr int kStages1 = (D == 128) ? 3 : 6;                       // HBM stream
+  static constexpr int kStages2 = (D == 128) ? (NPAD == 32 ? 3 : 2) : 4;    // L2 re-read
+  static constexpr int kTmemCols = 2 * kAcc * NPAD;                         // 256 or 512
   static constexpr int kBarBytes = 512;
-  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 2 * kQBytes + kBarBytes +
-                                    kGroupWarps * NPAD * 8 + NPAD * 8 + kGroupWarps * 32 * 8;
+  static constexpr int kSmemBytes = 1024 + (kStages1 + kStages2) * kStageBytes + 3 * kQBytes + kBarBytes +
+                                    4 * NPAD * 8 + NPAD * 8 + kGroupWarps * 32 * 8;
 };
 
 struct FusedBarriers {
-  uint64_t full[8];
-  uint64_t empty[8];
-  uint64_t q_full[2];
-  uint64_t q_empty[2];
-  uint64_t acc_full[16];
-  uint64_t acc_free[16];
+  uint64_t full1[6], empty1[6];
+  uint64_t full2[4], empty2[4];
+  uint64_t q1_full[2], q1_empty[2], q2_full[2], q2_empty[2];
+  uint64_t acc1_full[kAcc], acc1_empty[kAcc], acc2_full[kAcc], acc2_empty[kAcc];
   uint32_t tmem_base;
   int abort_flag;
+  int p1_done;                 // phases (this CTA took part in) whose pass 1 is published
+  int p2_done;                 // ... whose pass 2 is finished
 };
 static_assert(sizeof(FusedBarriers) <= 512, "barrier block");
 
 template <int ID>
 __device__ __forceinline__ void group_sync() { asm volatile("bar.sync %0, %1;" ::"n"(ID), "n"(kGroupWarps * 32) : "memory"); }
+
 
 __device__ __forceinline__ int ld_acquire(const int* p) {
   int v;
@@ -65,10 +70,27 @@ __device__ __forceinline__ void red_release_add(int* p, int v) {
   asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
+// Bounded wait until *flag (shared memory, written by another warp of the CTA) reaches `target`.
+__device__ __forceinline__ bool wait_smem_counter(volatile int* flag, int target, volatile int* abort_flag,
+                                                  WorkspaceHeader* hdr, int site) {
+  if (*flag >= target) return true;
+  const long long t0 = clock64();
+  unsigned spins = 0;
+  while (*flag < target) {
+    __nanosleep(64);
+    if ((++spins & 0x3Fu) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) {
+      *abort_flag = 1;
+      raise_status(hdr, FASTKV_ERR_DEVICE_TIMEOUT, site);
+      return false;
+    }
+  }
+  return true;
+}
+
 template <int GG>
-__device__ __forceinline__ void add_heads(const float (&pr)[32], float (&a_h)[8]) {
+__device__ __forceinline__ void add_heads(const float (&pr)[16], float (&a_h)[8]) {
 #pragma unroll
-  for (int x = 0; x < 32; ++x) a_h[x % GG] += pr[x];
+  for (int x = 0; x < 16; ++x) a_h[x % GG] += pr[x];
 }
 
 // what one CTA does in one phase
@@ -84,8 +106,7 @@ __device__ __forceinline__ PhaseWork phase_work(const FusedParams& p, int phase,
   w.L = p.cu_seqlens ? p.cu_seqlens[w.b + 1] - w.row0 : p.total_len;
   if (w.L < p.window) { w.t0 = 0; w.n = 0; w.nact = 0; return w; }
   const int ntiles = (w.L + kTileKeys - 1) / kTileKeys;
-  int per = (ntiles + ncta - 1) / ncta;
-  if (per > p.slots) per = p.slots;                 // host guarantees ntiles <= ncta * slots
+  const int per = (ntiles + ncta - 1) / ncta;
   w.nact = (ntiles + per - 1) / per;
   w.t0 = cta * per;
   w.n = max(0, min(per, ntiles - w.t0));
@@ -93,6 +114,10 @@ __device__ __forceinline__ PhaseWork phase_work(const FusedParams& p, int phase,
 }
 
 }  // namespace
+
+static_assert(FusedCfg<128, 32>::kSmemBytes <= 232448 && FusedCfg<128, 64>::kSmemBytes <= 232448 &&
+              FusedCfg<64, 32>::kSmemBytes <= 232448 && FusedCfg<64, 64>::kSmemBytes <= 232448,
+              "dynamic shared memory per CTA");
 
 template <int D, int NPAD>
 __global__ void __launch_bounds__(kFusedThreads, 1)
@@ -102,22 +127,34 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
-  uint8_t* smem_k = smem;
-  uint8_t* smem_q = smem + Cfg::kStages * Cfg::kStageBytes;           // two buffers of kQBytes
-  FusedBarriers* bars = reinterpret_cast<FusedBarriers*>(smem_q + 2 * Cfg::kQBytes);
-  float2* warp_stats = reinterpret_cast<float2*>(reinterpret_cast<uint8_t*>(bars) + Cfg::kBarBytes);
-  float2* norm = warp_stats + kGroupWarps * NPAD;                     // [NPAD] (row max, 1 / row sum)
-  float2* merge_buf = norm + NPAD;                                    // [128] partial merges
+  uint8_t* smem_k1 = smem;
+  uint8_t* smem_k2 = smem_k1 + Cfg::kStages1 * Cfg::kStageBytes;
+  uint8_t* smem_q1 = smem_k2 + Cfg::kStages2 * Cfg::kStageBytes;      // two buffers of kQBytes
+  uint8_t* smem_q2 = smem_q1 + 2 * Cfg::kQBytes;                      // one buffer of kQBytes
+  FusedBarriers* bars = reinterpret_cast<FusedBarriers*>(smem_q2 + Cfg::kQBytes);
+  float2* warp_stats = reinterpret_cast<float2*>(reinterpret_cast<uint8_t*>(bars) + Cfg::kBarBytes);   // [4][NPAD]
+  float2* norm = warp_stats + 4 * NPAD;                               // [NPAD] (row max, 1 / row sum)
+  float2* merge_buf = norm + NPAD;                                    // [256] partial merges
+  constexpr int CPW = NPAD / 2;                                       // accumulator columns per epilogue warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, ncta = gridDim.x;
   const int n_phases = p.batch * p.n_kv_heads;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < Cfg::kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&bars->q_full[i], 1); mbar_init(&bars->q_empty[i], 1); }
-    for (int i = 0; i < Cfg::kSlots; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_free[i], kGroupWarps); }
+    for (int s = 0; s < Cfg::kStages1; ++s) { mbar_init(&bars->full1[s], 1); mbar_init(&bars->empty1[s], 1); }
+    for (int s = 0; s < Cfg::kStages2; ++s) { mbar_init(&bars->full2[s], 1); mbar_init(&bars->empty2[s], 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bars->q1_full[i], 1); mbar_init(&bars->q1_empty[i], 1);
+      mbar_init(&bars->q2_full[i], 1); mbar_init(&bars->q2_empty[i], 1);
+    }
+    for (int i = 0; i < kAcc; ++i) {
+      mbar_init(&bars->acc1_full[i], 1); mbar_init(&bars->acc1_empty[i], kGroupWarps);   // every warp of the group
+      mbar_init(&bars->acc2_full[i], 1); mbar_init(&bars->acc2_empty[i], kGroupWarps);
+    }
     bars->abort_flag = 0;
+    bars->p1_done = 0;
+    bars->p2_done = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     tma_prefetch_desc(&tmap_k);
@@ -133,204 +170,185 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   const uint32_t tmem_base = bars->tmem_base;
   volatile int* abort_flag = &bars->abort_flag;
 
-  if (warp == 0) {
-    // ---------------- TMA producer ----------------
+  if (warp == 0 || warp == 2) {
+    // ---------------- TMA producers (warp 0: pipeline 1 from HBM, warp 2: pipeline 2 from L2) ----------------
     if (lane == 0) {
-      const uint64_t pol_stream = l2_policy_evict_first();
-      const uint64_t pol_keep = l2_policy_evict_last();
+      const bool second = warp == 2;
+      const uint64_t pol_k = second ? l2_policy_evict_first() : l2_policy_evict_last();
+      const uint64_t pol_q = l2_policy_evict_last();
+      uint8_t* const ring = second ? smem_k2 : smem_k1;
+      uint8_t* const qbuf = second ? smem_q2 : smem_q1;
+      uint64_t* const full = second ? bars->full2 : bars->full1;
+      uint64_t* const empty = second ? bars->empty2 : bars->empty1;
+      uint64_t* const q_full = second ? bars->q2_full : bars->q1_full;
+      uint64_t* const q_empty = second ? bars->q2_empty : bars->q1_empty;
+      const int stages = second ? Cfg::kStages2 : Cfg::kStages1;
+      const int nq = second ? 1 : 2;                     // Q buffers of the pipeline
       int it = 0, u = 0;
       bool ok = true;
       for (int phase = 0; ok && phase < n_phases; ++phase) {
         const PhaseWork w = phase_work(p, phase, cta, ncta);
         if (w.n == 0) continue;
-        const int h = u & 1;
-        if (u >= 2) ok = mbar_wait_bounded(&bars->q_empty[h], ((u >> 1) - 1) & 1, abort_flag, p.hdr, SITE_FUSED_Q_EMPTY);
+        // pipeline 2 re-reads what pipeline 1 of this CTA has finished with; pipeline 1 stays close
+        // enough ahead for those tiles to be still in L2
+        if (second) ok = wait_smem_counter(&bars->p1_done, u + 1, abort_flag, p.hdr, SITE_FUSED_P1_DONE);
+        else if (u >= p.max_lead) ok = wait_smem_counter(&bars->p2_done, u - p.max_lead + 1, abort_flag, p.hdr, SITE_FUSED_P2_DONE);
+        const int h = u % nq;
+        if (ok && u >= nq) ok = mbar_wait_bounded(&q_empty[h], ((u / nq) - 1) & 1, abort_flag, p.hdr, SITE_FUSED_Q_EMPTY);
         if (!ok) break;
         const int q_row0 = (p.q_layout == FASTKV_Q_WINDOW) ? w.b * p.window : w.row0 + w.L - p.window;
-        mbar_arrive_expect_tx(&bars->q_full[h], Cfg::KH * p.n_rows * 128);
+        mbar_arrive_expect_tx(&q_full[h], Cfg::KH * p.n_rows * 128);
         for (int c = 0; c < Cfg::KH; ++c)
-          tma_load_3d(smem_q + h * Cfg::kQBytes + c * NPAD * 128, &tmap_q, &bars->q_full[h], c * 64,
-                      w.g * p.group, q_row0, pol_keep);
+          tma_load_3d(qbuf + h * Cfg::kQBytes + c * NPAD * 128, &tmap_q, &q_full[h], c * 64, w.g * p.group, q_row0,
+                      pol_q);
         for (int i = 0; i < w.n; ++i, ++it) {
-          const int s = it % Cfg::kStages;
-          ok = mbar_wait_bounded(&bars->empty[s], ((it / Cfg::kStages) & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_EMPTY);
+          const int s = it % stages;
+          ok = mbar_wait_bounded(&empty[s], ((it / stages) & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_EMPTY);
           if (!ok) break;
-          mbar_arrive_expect_tx(&bars->full[s], Cfg::kStageBytes);
+          mbar_arrive_expect_tx(&full[s], Cfg::kStageBytes);
           for (int c = 0; c < Cfg::KH; ++c)
-            tma_load_3d(smem_k + s * Cfg::kStageBytes + c * kHalfBytes, &tmap_k, &bars->full[s], c * 64, w.g,
-                        w.row0 + (w.t0 + i) * kTileKeys, pol_stream);
+            tma_load_3d(ring + s * Cfg::kStageBytes + c * kHalfBytes, &tmap_k, &full[s], c * 64, w.g,
+                        w.row0 + (w.t0 + i) * kTileKeys, pol_k);
         }
         ++u;
       }
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer: accumulators form a ring of kSlots tensor-memory slots ----------------
+  } else if (warp == 1 || warp == 3) {
+    // ---------------- MMA issuers (warp 1: pipeline 1, warp 3: pipeline 2) ----------------
     if (lane == 0) {
+      const bool second = warp == 3;
       constexpr uint32_t idesc = umma_idesc_bf16_f32(kTileKeys, NPAD);
-      int it = 0, u = 0, seq = 0;
+      uint8_t* const ring = second ? smem_k2 : smem_k1;
+      uint8_t* const qbuf = second ? smem_q2 : smem_q1;
+      uint64_t* const full = second ? bars->full2 : bars->full1;
+      uint64_t* const empty = second ? bars->empty2 : bars->empty1;
+      uint64_t* const q_full = second ? bars->q2_full : bars->q1_full;
+      uint64_t* const q_empty = second ? bars->q2_empty : bars->q1_empty;
+      uint64_t* const acc_full = second ? bars->acc2_full : bars->acc1_full;
+      uint64_t* const acc_empty = second ? bars->acc2_empty : bars->acc1_empty;
+      const int stages = second ? Cfg::kStages2 : Cfg::kStages1;
+      const int nq = second ? 1 : 2;
+      const uint32_t acc_base = tmem_base + (second ? kAcc * NPAD : 0);
+      int it = 0, u = 0;
       bool ok = true;
       for (int phase = 0; ok && phase < n_phases; ++phase) {
         const PhaseWork w = phase_work(p, phase, cta, ncta);
         if (w.n == 0) continue;
-        const int h = u & 1;
-        ok = mbar_wait_bounded(&bars->q_full[h], (u >> 1) & 1, abort_flag, p.hdr, SITE_FUSED_Q_FULL);
+        const int h = u % nq;
+        ok = mbar_wait_bounded(&q_full[h], (u / nq) & 1, abort_flag, p.hdr, SITE_FUSED_Q_FULL);
         if (!ok) break;
-        const uint32_t q_addr = smem_u32(smem_q + h * Cfg::kQBytes);
+        const uint32_t q_addr = smem_u32(qbuf + h * Cfg::kQBytes);
         for (int i = 0; i < w.n; ++i, ++it) {
-          const int s = it % Cfg::kStages, slot = (seq + i) % Cfg::kSlots, use = (seq + i) / Cfg::kSlots;
-          ok = mbar_wait_bounded(&bars->acc_free[slot], (use & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_ACC_FREE) &&
-               mbar_wait_bounded(&bars->full[s], (it / Cfg::kStages) & 1, abort_flag, p.hdr, SITE_FUSED_FULL);
+          const int s = it % stages, a = it % kAcc;
+          ok = mbar_wait_bounded(&acc_empty[a], ((it / kAcc) & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_ACC_FREE) &&
+               mbar_wait_bounded(&full[s], (it / stages) & 1, abort_flag, p.hdr, SITE_FUSED_FULL);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t k_addr = smem_u32(smem_k + s * Cfg::kStageBytes);
+          const uint32_t k_addr = smem_u32(ring + s * Cfg::kStageBytes);
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
             const uint64_t adesc = umma_desc_k_sw128(k_addr + (kk >> 2) * kHalfBytes + (kk & 3) * 32);
             const uint64_t bdesc = umma_desc_k_sw128(q_addr + (kk >> 2) * NPAD * 128 + (kk & 3) * 32);
-            tc_mma_bf16(tmem_base + slot * NPAD, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
+            tc_mma_bf16(acc_base + a * NPAD, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
           }
-          tc_commit(&bars->empty[s]);
-          tc_commit(&bars->acc_full[slot]);
+          tc_commit(&empty[s]);
+          tc_commit(&acc_full[a]);
         }
-        if (ok) tc_commit(&bars->q_empty[h]);
-        seq += w.n + 1;                                  // the phase's tiles plus its statistics slot
+        if (ok) tc_commit(&q_empty[h]);
         ++u;
       }
     }
-  } else if (warp < 2 + kGroupWarps) {
-    // ---------------- group A: pass 1 ----------------
-    // Per tile: e = exp2(s - m) with a per-(lane, row) reference m, written back over the logits;
-    // l += e.  m is the row's first logit and moves only when a logit exceeds it by more than the
-    // slack (rare); then l and the e already stored for the phase's earlier tiles are rescaled,
-    // so that at the end of the phase every stored e of a lane is relative to its final m.
-    const int quarter = warp & 3;
+  } else if (warp < kCtrlWarps + kGroupWarps) {
+    // ---------------- group A: pass 1, running (max, sum of exp2) per query row; publish per phase ----------------
+    // 8 warps: warp (quarter, half) owns tensor-memory lanes 32 * quarter .. +31 (one key per lane)
+    // and the accumulator columns (query rows) half * CPW .. +CPW-1.
+    const int gw = warp - kCtrlWarps;
+    const int quarter = warp & 3, half = gw >> 2;
     const int key_in_tile = quarter * 32 + lane;
-    const int at = threadIdx.x - 64;                    // 0..127 within the group
+    const int at = threadIdx.x - kCtrlWarps * 32;       // 0..255 within the group
     const int n_rows = p.n_rows, G = p.group;
-    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-    int seq = 0;
+    const int col0 = half * CPW;                         // first query row of this warp
+    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + col0;
+    int it = 0, u = 0;
     bool ok = true;
     for (int phase = 0; ok && phase < n_phases; ++phase) {
       const PhaseWork w = phase_work(p, phase, cta, ncta);
       if (w.n == 0) continue;
-      float m[NPAD], l[NPAD];
+      float m[CPW], l[CPW];
+#pragma unroll
+      for (int n = 0; n < CPW; ++n) { m[n] = -INFINITY; l[n] = 0.0f; }
       const int win_start = w.L - p.window;
-      for (int i = 0; i < w.n; ++i) {
-        const int slot = (seq + i) % Cfg::kSlots, use = (seq + i) / Cfg::kSlots;
-        ok = mbar_wait_bounded(&bars->acc_full[slot], use & 1, abort_flag, p.hdr, SITE_FUSED_ACC_FULL);
+      for (int i = 0; i < w.n; ++i, ++it) {
+        const int a = it % kAcc;
+        ok = mbar_wait_bounded(&bars->acc1_full[a], (it / kAcc) & 1, abort_flag, p.hdr, SITE_FUSED_ACC_FULL);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after_sync();
         const int key = (w.t0 + i) * kTileKeys + key_in_tile;
         const bool tile_unmasked = (w.t0 + i + 1) * kTileKeys <= win_start;
 #pragma unroll
-        for (int c = 0; c < NPAD / 32; ++c) {
-          float e[32];
-          const uint32_t taddr = lane_base + slot * NPAD + c * 32;
-          tmem_ld_32x32(taddr, e);
-          const int n_valid = n_rows - c * 32;
-          uint32_t visible = 0xffffffffu;                // causal: key i <= t_j, j = n / G
-          if (!tile_unmasked) {
-            visible = 0;
+        for (int c = 0; c < CPW / 16; ++c) {
+          float acc[16];
+          tmem_ld_32x16(lane_base + a * NPAD + c * 16, acc);
+          if (c == CPW / 16 - 1) {                       // this warp's part of the accumulator is in registers
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->acc1_empty[a]);
+          }
+          const int n_valid = n_rows - col0 - c * 16;
+          if (tile_unmasked) {
+            if (i == 0) stats_init_unmasked<16>(acc, m + c * 16, l + c * 16, p.scale_log2, n_valid);
+            else stats_update_unmasked<16>(acc, m + c * 16, l + c * 16, p.scale_log2, n_valid);
+          } else {
+            uint32_t visible = 0;                        // causal: key i <= t_j, j = n / G
             if (key < w.L) {
 #pragma unroll
-              for (int x = 0; x < 32; ++x)
-                if (x < n_valid && key <= win_start + (c * 32 + x) / G) visible |= 1u << x;
+              for (int x = 0; x < 16; ++x)
+                if (x < n_valid && key <= win_start + (col0 + c * 16 + x) / G) visible |= 1u << x;
             }
+            stats_update_masked<16>(acc, m + c * 16, l + c * 16, p.scale_log2, n_valid, visible);
           }
-          float* const mc = m + c * 32;
-          float* const lc = l + c * 32;
-          if (i == 0) {
-#pragma unroll
-            for (int x = 0; x < 32; ++x) {
-              const bool vis = (visible >> x) & 1u;
-              mc[x] = vis ? e[x] * p.scale_log2 : -INFINITY;
-              e[x] = vis ? 1.0f : 0.0f;
-              lc[x] = e[x];
-            }
-          } else {
-            bool need = false;                           // s - m is +inf while m = -inf
-#pragma unroll
-            for (int x = 0; x < 32; ++x)
-              need |= (x < n_valid) && ((visible >> x) & 1u) && (fmaf(e[x], p.scale_log2, -mc[x]) > kLazyMaxSlackLog2);
-            if (__any_sync(0xffffffffu, need)) {         // rare: some reference moves up to its new logit
-              float fac[32];
-#pragma unroll
-              for (int x = 0; x < 32; ++x) {
-                const float sx = e[x] * p.scale_log2;
-                const bool mv = (x < n_valid) && ((visible >> x) & 1u) && (sx - mc[x] > kLazyMaxSlackLog2);
-                fac[x] = (mv && mc[x] != -INFINITY) ? ex2(mc[x] - sx) : 1.0f;      // 2^(m_old - m_new)
-                mc[x] = mv ? sx : mc[x];
-                lc[x] *= fac[x];
-              }
-              for (int j = 0; j < i; ++j) {              // earlier tiles of the phase: e *= 2^(m_old - m_new)
-                const uint32_t tj = lane_base + ((seq + j) % Cfg::kSlots) * NPAD + c * 32;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                  float old[8];
-                  tmem_ld_32x8(tj + q * 8, old);
-#pragma unroll
-                  for (int x = 0; x < 8; ++x) old[x] *= fac[q * 8 + x];
-                  tmem_st_32x8(tj + q * 8, old);
-                }
-              }
-            }
-#pragma unroll
-            for (int x = 0; x < 32; ++x) {
-              e[x] = ((visible >> x) & 1u) ? ex2(fmaf(e[x], p.scale_log2, -mc[x])) : 0.0f;
-              lc[x] += e[x];
-            }
-          }
-          tmem_st_32x32(taddr, e);
         }
       }
       if (!ok) break;
-      // the lane's final references go into the phase's statistics slot for group B
-      const int sslot = (seq + w.n) % Cfg::kSlots, suse = (seq + w.n) / Cfg::kSlots;
-      ok = mbar_wait_bounded(&bars->acc_free[sslot], (suse & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_ACC_FREE);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after_sync();
+      // lanes -> warp: after the butterfly lanes r and r + 16 hold row col0 + c * 16 + r in entry c * 16
 #pragma unroll
-      for (int c = 0; c < NPAD / 32; ++c)
-        tmem_st_32x32(lane_base + sslot * NPAD + c * 32, *reinterpret_cast<const float(*)[32]>(m + c * 32));
-      tmem_wait_st();
-      tc_fence_before_sync();
-      // lanes -> warp: after the butterfly lane r holds row c * 32 + r in entry c * 32
-#pragma unroll
-      for (int c = 0; c < NPAD / 32; ++c) {
-        stats_transpose_merge(m + c * 32, l + c * 32, lane);
-        warp_stats[quarter * NPAD + c * 32 + lane] = make_float2(m[c * 32], l[c * 32]);
+      for (int c = 0; c < CPW / 16; ++c) {
+        stats_transpose_merge<16>(m + c * 16, l + c * 16, lane);
+        if (lane < 16) warp_stats[quarter * NPAD + col0 + c * 16 + lane] = make_float2(m[c * 16], l[c * 16]);
       }
       group_sync<1>();
-      if (at < NPAD) {                                   // warps -> CTA, publish
+      if (at < NPAD) {                                   // lane quarters -> CTA, publish
         float mm = -INFINITY, ll = 0.0f;
 #pragma unroll
-        for (int q = 0; q < kGroupWarps; ++q) merge_stats(mm, ll, warp_stats[q * NPAD + at].x, warp_stats[q * NPAD + at].y);
+        for (int q = 0; q < 4; ++q) merge_stats(mm, ll, warp_stats[q * NPAD + at].x, warp_stats[q * NPAD + at].y);
         p.partial[(static_cast<size_t>(phase) * ncta + cta) * NPAD + at] = make_float2(mm, ll);
       }
       group_sync<1>();                                   // also: warp_stats may be rewritten next phase
+      ++u;
       if (at == 0) {
         red_release_add(p.counters + phase, 1);          // release: cumulative over the barrier
-        mbar_arrive(&bars->acc_full[sslot]);             // keeps this slot's full/free parities in step
+        bars->p1_done = u;                               // pipeline 2 may re-read this phase's tiles
       }
-      seq += w.n + 1;
     }
   } else {
-    // ---------------- group B: pass 2 ----------------
-    // Once every CTA of the phase has published: merge the statistics into (M_r, 1 / l_r), turn the
-    // lane's references into factors f = 2^(m - M_r) / l_r, and sum e * f over the window rows (and
-    // the group) of each key.  No exponential per logit here.
-    const int quarter = warp & 3;
+    // ---------------- group B: pass 2, normalise and sum over window rows / group ----------------
+    // Same (quarter, half) split as group A; each half writes its partial sums to its own plane of
+    // a_out, and the pooling kernel adds the two planes.
+    const int gw = warp - kCtrlWarps - kGroupWarps;
+    const int quarter = warp & 3, half = gw >> 2;
     const int key_in_tile = quarter * 32 + lane;
-    const int bt = threadIdx.x - 64 - kGroupWarps * 32;   // 0..127 within the group
+    const int bt = threadIdx.x - (kCtrlWarps + kGroupWarps) * 32;   // 0..255 within the group
     const int n_rows = p.n_rows, G = p.group;
-    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    const int col0 = half * CPW;
+    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + kAcc * NPAD + col0;
     constexpr int kParts = kGroupWarps * 32 / NPAD;
-    int seq = 0;
-    for (int phase = 0; phase < n_phases; ++phase) {
+    int it = 0, u = 0;
+    bool ok = true;
+    for (int phase = 0; ok && phase < n_phases; ++phase) {
       const PhaseWork w = phase_work(p, phase, cta, ncta);
       if (w.n == 0) continue;
+      // every CTA that owns tiles of this phase has published its statistics?
       if (bt == 0) {
         const int* ctr = p.counters + phase;
         if (ld_acquire(ctr) < w.nact) {
@@ -358,45 +376,44 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         norm[bt] = (bt < n_rows && ll > 0.0f) ? make_float2(mm, 1.0f / ll) : make_float2(0.0f, 0.0f);
       }
       group_sync<2>();
-      tc_fence_after_sync();
-      const int sslot = (seq + w.n) % Cfg::kSlots;
-      float f[NPAD];
+      float nm[CPW], nil[CPW];                           // -(row max) and 1 / (row sum) of this warp's rows
 #pragma unroll
-      for (int c = 0; c < NPAD / 32; ++c) {
-        float mref[32];
-        tmem_ld_32x32(lane_base + sslot * NPAD + c * 32, mref);
-#pragma unroll
-        for (int x = 0; x < 32; ++x) {
-          const float2 st = norm[c * 32 + x];
-          f[c * 32 + x] = (c * 32 + x < n_rows) ? ex2(mref[x] - st.x) * st.y : 0.0f;   // m = -inf gives 0
-        }
-      }
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->acc_free[sslot]);
-      for (int i = 0; i < w.n; ++i) {
-        const int slot = (seq + i) % Cfg::kSlots;
+      for (int n = 0; n < CPW; ++n) { const float2 st = norm[col0 + n]; nm[n] = -st.x; nil[n] = st.y; }
+      const int win_start = w.L - p.window;
+      for (int i = 0; i < w.n; ++i, ++it) {
+        const int a = it % kAcc;
+        ok = mbar_wait_bounded(&bars->acc2_full[a], (it / kAcc) & 1, abort_flag, p.hdr, SITE_FUSED_ACC_FULL);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
         const int key = (w.t0 + i) * kTileKeys + key_in_tile;
+        const bool tile_unmasked = (w.t0 + i + 1) * kTileKeys <= win_start;
         float a_g = 0.0f;
         float a_h[8];                                    // per query head of the group (G in {1,2,4,8})
 #pragma unroll
         for (int q = 0; q < 8; ++q) a_h[q] = 0.0f;
 #pragma unroll
-        for (int c = 0; c < NPAD / 32; ++c) {
-          float pr[32];
-          tmem_ld_32x32(lane_base + slot * NPAD + c * 32, pr);
-          if (c == NPAD / 32 - 1) {                      // the slot is in registers: hand it back
+        for (int c = 0; c < CPW / 16; ++c) {
+          float pr[16];
+          tmem_ld_32x16(lane_base + a * NPAD + c * 16, pr);
+          if (c == CPW / 16 - 1) {                       // this warp's part of the accumulator is in registers
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->acc_free[slot]);
+            if (lane == 0) mbar_arrive(&bars->acc2_empty[a]);
           }
-          const int n_valid = n_rows - c * 32;
+          const int n_valid = n_rows - col0 - c * 16;
 #pragma unroll
-          for (int x = 0; x < 32; ++x) pr[x] = (x < n_valid) ? pr[x] * f[c * 32 + x] : 0.0f;
+          for (int x = 0; x < 16; ++x)
+            pr[x] = (x < n_valid) ? ex2(fmaf(pr[x], p.scale_log2, nm[c * 16 + x])) * nil[c * 16 + x] : 0.0f;
+          if (!tile_unmasked) {                          // causal: key i <= t_j, j = n / G
+#pragma unroll
+            for (int x = 0; x < 16; ++x)
+              if (x < n_valid && key > win_start + (col0 + c * 16 + x) / G) pr[x] = 0.0f;
+          }
           if (!p.per_head) {
 #pragma unroll
-            for (int x = 0; x < 32; x += 4) a_g += (pr[x] + pr[x + 1]) + (pr[x + 2] + pr[x + 3]);
-          } else {                                       // row n = j * G + hl and G divides 32
+            for (int x = 0; x < 16; x += 4) a_g += (pr[x] + pr[x + 1]) + (pr[x + 2] + pr[x + 3]);
+          } else {                                       // row n = j * G + hl and G divides 16
             switch (G) {
               case 1: add_heads<1>(pr, a_h); break;
               case 2: add_heads<2>(pr, a_h); break;
@@ -405,18 +422,21 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             }
           }
         }
+        // each column half writes its own plane of partial sums; the pooling kernel adds the two
         if (key < w.L) {
+          float* const plane = p.a_out + static_cast<size_t>(half) * p.plane_stride;
           if (p.per_head) {
 #pragma unroll
             for (int q = 0; q < 8; ++q)
-              if (q < G) p.a_out[static_cast<size_t>(w.g * G + q) * p.ld_a + w.row0 + key] = a_h[q];
+              if (q < G) plane[static_cast<size_t>(w.g * G + q) * p.ld_a + w.row0 + key] = a_h[q];
           } else {
-            p.a_out[static_cast<size_t>(w.g) * p.ld_a + w.row0 + key] = a_g;
+            plane[static_cast<size_t>(w.g) * p.ld_a + w.row0 + key] = a_g;
           }
         }
       }
       group_sync<2>();                                   // norm / merge_buf are rewritten next phase
-      seq += w.n + 1;
+      ++u;
+      if (bt == 0) bars->p2_done = u;                    // lets pipeline 1 move further ahead
     }
   }
 
@@ -446,7 +466,8 @@ __global__ void __launch_bounds__(kPoolThreads) pool_rows_kernel(const PoolRowsP
   for (int item = threadIdx.x; item < rows * span; item += blockDim.x) {
     const int row = item / span, o = item - row * span;
     const int key = k0 - r + o;
-    sm[item] = (key >= 0 && key < L) ? __ldg(p.a + static_cast<size_t>(row) * p.ld_a + row0 + key) : 0.0f;
+    const float* src = p.a + static_cast<size_t>(row) * p.ld_a + row0 + key;
+    sm[item] = (key >= 0 && key < L) ? __ldg(src) + __ldg(src + p.plane_stride) : 0.0f;
   }
   __syncthreads();
   const float inv_p = 1.0f / static_cast<float>(p.pool_kernel);
@@ -477,7 +498,6 @@ __global__ void __launch_bounds__(kPoolThreads) pool_rows_kernel(const PoolRowsP
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
-int fused_slots(int npad) { return 512 / npad - 1; }   // one slot per phase carries the lanes' references
 
 template <int D, int NPAD>
 static cudaError_t launch_fused_t(const CUtensorMap& tk, const CUtensorMap& tq, const FusedParams& p, int grid,
