@@ -3,8 +3,8 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
-One "step" is one pass of the whole hot path (fastkv_score, fastkv_select_kv, fastkv_select_tsp,
-fastkv_compact) over one layer of synthetic, seeded input.  The default workload is the
+One "step" is one pass of the whole hot path (fastkv_score, fastkv_select = select_kv + select_tsp in
+one launch, fastkv_compact) over one layer of synthetic, seeded input.  The default workload is the
 Llama-3.1-8B-shaped layer at L = 131072 with Token-Selective Propagation (KV retention 10 %, TSP
 rate 20 %).  With N > 1 (torchrun, one rank per GPU) every rank runs its own layer of the same
 shape -- the path partitions over independent layers / requests, so there is no collective on the
@@ -250,11 +250,9 @@ def main() -> None:
         B.fastkv_score(shape, q, k, s_kv, s_tsp, ws, stream)
         if events is not None:
             events[1].record(stream)
-        B.fastkv_select_kv(shape, s_kv, b_kv, idx_kv, ws, stream)
+        B.fastkv_select(shape, s_kv, b_kv, idx_kv, s_tsp, b_tsp, idx_tsp, ws, stream)   # select_kv + select_tsp
         if events is not None:
             events[2].record(stream)
-        B.fastkv_select_tsp(shape, s_tsp, b_tsp, idx_tsp, ws, stream)
-        if events is not None:
             events[3].record(stream)
         B.fastkv_compact(shape, idx_kv, b_kv, idx_tsp, b_tsp, k, v, hid, pos, k_out, v_out, hid_out, pos_out, ws,
                          stream)
@@ -364,8 +362,7 @@ def main() -> None:
                           "frac_of_measured": step_gbs / peaks["hbm_gbs"],
                           "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
                           "rows_once_gbs": ab["step_min"] / (ms_per_step * 1e-3) / 1e9},
-        "calls_ms": {"fastkv_score": call_ms[0], "fastkv_select_kv": call_ms[1], "fastkv_select_tsp": call_ms[2],
-                     "fastkv_compact": call_ms[3]},
+        "calls_ms": {"fastkv_score": call_ms[0], "fastkv_select": call_ms[1], "fastkv_compact": call_ms[3]},
         "calls_gbs": {"fastkv_score": ab["score"] / (call_ms[0] * 1e-3) / 1e9},
     }
     if not args.no_cpu_baseline:

@@ -130,6 +130,15 @@ int fastkv_select_tsp(const fastkv_shape* shape, const float* scores_tsp, const 
                       int32_t* idx_tsp, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Both selections of a TSP layer in one launch (KVCompress and HiddenCompress, App. B.1): exactly
+ * what fastkv_select_kv followed by fastkv_select_tsp produce, but the nine problems of a layer
+ * (one per KV head plus the layer-level one) run side by side instead of one call after the other.
+ */
+int fastkv_select(const fastkv_shape* shape, const float* scores_kv, const fastkv_budget* kv, int32_t* idx_kv,
+                  const float* scores_tsp, const fastkv_budget* tsp, int32_t* idx_tsp, void* workspace,
+                  size_t workspace_bytes, void* stream);
+
+/*
  * Compaction (Alg. 1: C <- update(K, V); reduced hidden states x).  Byte copies:
  *   k_out[g, j, :]   = k[cu_seqlens[b] + idx_kv[g, j], g, :]     [n_kv_heads, kv.total, head_dim]
  *   v_out likewise                                               (v, v_out may both be NULL)

@@ -20,7 +20,7 @@ POOL_AVG, POOL_MAX = 0, 1
 GROUP_THEN_POOL, POOL_THEN_GROUP = 0, 1
 Q_FULL, Q_WINDOW = 0, 1
 
-EXPORTS = ["fastkv_workspace_bytes", "fastkv_score", "fastkv_select_kv", "fastkv_select_tsp",
+EXPORTS = ["fastkv_workspace_bytes", "fastkv_score", "fastkv_select_kv", "fastkv_select_tsp", "fastkv_select",
            "fastkv_compact", "fastkv_device_status", "fastkv_layer_host_arena_bytes",
            "fastkv_layer_host", "fastkv_score_static", "fastkv_status_string", "fastkv_last_error",
            "fastkv_kernel_launches"]
@@ -71,6 +71,7 @@ def _load():
         lib.fastkv_score.argtypes = [ps, vp, vp, vp, vp, vp, sz, vp]
         lib.fastkv_select_kv.argtypes = [ps, vp, pb, vp, vp, sz, vp]
         lib.fastkv_select_tsp.argtypes = [ps, vp, pb, vp, vp, sz, vp]
+        lib.fastkv_select.argtypes = [ps, vp, pb, vp, vp, pb, vp, vp, sz, vp]
         lib.fastkv_compact.argtypes = [ps, vp, pb, vp, pb, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.fastkv_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
         lib.fastkv_layer_host_arena_bytes.argtypes = [ps, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(sz)]
@@ -80,7 +81,7 @@ def _load():
         lib.fastkv_last_error.restype = ctypes.c_char_p
         lib.fastkv_kernel_launches.restype = ctypes.c_int64
         lib.fastkv_score_static.argtypes = [ps, vp, vp, vp, vp, vp]
-        for fn in EXPORTS[:9]:
+        for fn in EXPORTS[:10]:
             getattr(lib, fn).restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -163,6 +164,13 @@ def fastkv_select_tsp(shape: Shape, scores_tsp, budget: Budget, idx_tsp, workspa
     _check(_load().fastkv_select_tsp(ctypes.byref(shape), _p(scores_tsp), ctypes.byref(budget), _p(idx_tsp),
                                      _p(workspace), workspace.numel() * workspace.element_size(),
                                      _stream(stream)), "fastkv_select_tsp")
+
+
+def fastkv_select(shape: Shape, scores_kv, kv: Budget, idx_kv, scores_tsp, tsp: Budget, idx_tsp, workspace,
+                  stream=None) -> None:
+    _check(_load().fastkv_select(ctypes.byref(shape), _p(scores_kv), ctypes.byref(kv), _p(idx_kv), _p(scores_tsp),
+                                 ctypes.byref(tsp), _p(idx_tsp), _p(workspace),
+                                 workspace.numel() * workspace.element_size(), _stream(stream)), "fastkv_select")
 
 
 def fastkv_compact(shape: Shape, idx_kv, kv: Optional[Budget], idx_tsp, tsp: Optional[Budget], k, v, hidden,

@@ -339,21 +339,24 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
   return FASTKV_OK;
 }
 
-static int select_common(const fastkv_shape* shape, const float* scores, const fastkv_budget* budget,
-                         int32_t* idx, int n_rows, void* workspace, size_t workspace_bytes, void* stream_,
-                         const char* name) {
-  int rc = check_shape(shape, false);
-  if (rc) return rc;
+static int fill_select_set(const fastkv_shape* shape, const float* scores, const fastkv_budget* budget, int32_t* idx,
+                           int n_rows, const char* name, SelectSet* set) {
   if (scores == nullptr || idx == nullptr) return fail(FASTKV_ERR_INVALID_ARG, "%s: scores and idx are required", name);
-  if ((rc = check_budget(shape, budget, name))) return rc;
-  if ((rc = check_workspace(workspace, workspace_bytes, sizeof(WorkspaceHeader)))) return rc;
+  int rc = check_budget(shape, budget, name);
+  if (rc) return rc;
+  set->scores = scores; set->ld_scores = shape->total_len; set->idx = idx; set->ld_idx = budget->total;
+  set->cu_k = budget->cu_k; set->k_uniform = budget->k; set->n_rows = n_rows;
+  return FASTKV_OK;
+}
+
+static int launch_select_sets(const fastkv_shape* shape, SelectParams& p, void* workspace, size_t workspace_bytes,
+                              void* stream_) {
+  int rc = check_workspace(workspace, workspace_bytes, sizeof(WorkspaceHeader));
+  if (rc) return rc;
   if ((rc = check_device())) return rc;
-  SelectParams p;
-  p.scores = scores; p.ld_scores = shape->total_len; p.idx = idx; p.ld_idx = budget->total;
-  p.cu_seqlens = shape->cu_seqlens; p.cu_k = budget->cu_k; p.k_uniform = budget->k;
-  p.total_len = shape->total_len; p.window = shape->window; p.force_window = shape->force_window;
-  p.hdr = static_cast<WorkspaceHeader*>(workspace);
-  cudaError_t e = launch_select(p, n_rows, shape->batch, shape->max_len, static_cast<cudaStream_t>(stream_));
+  p.cu_seqlens = shape->cu_seqlens; p.total_len = shape->total_len; p.window = shape->window;
+  p.force_window = shape->force_window; p.hdr = static_cast<WorkspaceHeader*>(workspace);
+  cudaError_t e = launch_select(p, shape->batch, shape->max_len, static_cast<cudaStream_t>(stream_));
   if (e != cudaSuccess) return cuda_fail(e, "select_topk_kernel launch");
   ++g_launches;
   return FASTKV_OK;
@@ -361,13 +364,34 @@ static int select_common(const fastkv_shape* shape, const float* scores, const f
 
 int fastkv_select_kv(const fastkv_shape* shape, const float* scores_kv, const fastkv_budget* budget,
                      int32_t* idx_kv, void* workspace, size_t workspace_bytes, void* stream) {
-  return select_common(shape, scores_kv, budget, idx_kv, shape ? shape->n_kv_heads : 0, workspace,
-                       workspace_bytes, stream, "select_kv");
+  int rc = check_shape(shape, false);
+  if (rc) return rc;
+  SelectParams p;
+  memset(&p, 0, sizeof p);
+  if ((rc = fill_select_set(shape, scores_kv, budget, idx_kv, shape->n_kv_heads, "select_kv", &p.set[0]))) return rc;
+  return launch_select_sets(shape, p, workspace, workspace_bytes, stream);
 }
 
 int fastkv_select_tsp(const fastkv_shape* shape, const float* scores_tsp, const fastkv_budget* budget,
                       int32_t* idx_tsp, void* workspace, size_t workspace_bytes, void* stream) {
-  return select_common(shape, scores_tsp, budget, idx_tsp, 1, workspace, workspace_bytes, stream, "select_tsp");
+  int rc = check_shape(shape, false);
+  if (rc) return rc;
+  SelectParams p;
+  memset(&p, 0, sizeof p);
+  if ((rc = fill_select_set(shape, scores_tsp, budget, idx_tsp, 1, "select_tsp", &p.set[0]))) return rc;
+  return launch_select_sets(shape, p, workspace, workspace_bytes, stream);
+}
+
+int fastkv_select(const fastkv_shape* shape, const float* scores_kv, const fastkv_budget* kv, int32_t* idx_kv,
+                  const float* scores_tsp, const fastkv_budget* tsp, int32_t* idx_tsp, void* workspace,
+                  size_t workspace_bytes, void* stream) {
+  int rc = check_shape(shape, false);
+  if (rc) return rc;
+  SelectParams p;
+  memset(&p, 0, sizeof p);
+  if ((rc = fill_select_set(shape, scores_kv, kv, idx_kv, shape->n_kv_heads, "select (kv)", &p.set[0]))) return rc;
+  if ((rc = fill_select_set(shape, scores_tsp, tsp, idx_tsp, 1, "select (tsp)", &p.set[1]))) return rc;
+  return launch_select_sets(shape, p, workspace, workspace_bytes, stream);
 }
 
 int fastkv_compact(const fastkv_shape* shape, const int32_t* idx_kv, const fastkv_budget* kv,
@@ -517,8 +541,11 @@ int fastkv_layer_host(const fastkv_shape* shape, int32_t k_kv, int32_t k_tsp, co
   fastkv_budget bkv = {k_kv, k_kv * s.batch, nullptr}, btsp = {k_tsp, k_tsp * s.batch, nullptr};
   int32_t* d_idx_kv = reinterpret_cast<int32_t*>(d + a.idx_kv);
   int32_t* d_idx_tsp = reinterpret_cast<int32_t*>(d + a.idx_tsp);
-  if ((rc = fastkv_select_kv(&s, scores_kv, &bkv, d_idx_kv, ws, a.ws_bytes, stream))) return rc;
-  if (k_tsp && (rc = fastkv_select_tsp(&s, scores_tsp, &btsp, d_idx_tsp, ws, a.ws_bytes, stream))) return rc;
+  if (k_tsp) {
+    if ((rc = fastkv_select(&s, scores_kv, &bkv, d_idx_kv, scores_tsp, &btsp, d_idx_tsp, ws, a.ws_bytes, stream))) return rc;
+  } else if ((rc = fastkv_select_kv(&s, scores_kv, &bkv, d_idx_kv, ws, a.ws_bytes, stream))) {
+    return rc;
+  }
   if ((rc = fastkv_compact(&s, d_idx_kv, &bkv, k_tsp ? d_idx_tsp : nullptr, k_tsp ? &btsp : nullptr, d + a.k, d + a.v,
                            k_tsp ? d + a.hidden : nullptr, k_tsp ? reinterpret_cast<const int32_t*>(d + a.pos) : nullptr,
                            d + a.k_out, d + a.v_out, k_tsp ? d + a.hidden_out : nullptr,

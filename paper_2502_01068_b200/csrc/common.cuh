@@ -47,6 +47,14 @@ __device__ __forceinline__ void raise_status(WorkspaceHeader* hdr, int status, i
   if (hdr != nullptr && atomicCAS(&hdr->status, 0, status) == 0) hdr->site = site;
 }
 
+// ---- programmatic dependent launch -----------------------------------------------------------
+// Kernels of one layer step are chained on a stream.  A kernel launched with the programmatic
+// stream serialization attribute may start while its predecessor drains; pdl_wait() blocks until
+// the predecessor has completed and its writes are visible (a no-op for an ordinary launch), and
+// pdl_launch_dependents() tells the scheduler that the successor may be brought up.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- shared-memory addresses ---------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -380,6 +388,12 @@ __device__ __forceinline__ float2 merge_partials(const float2* part, int npad, i
     for (int j = 0; j < 20; ++j) merge_stats(m, l, v[j].x, v[j].y);
   }
   return make_float2(m, l);
+}
+
+// Launch configuration shared by the kernels that follow another kernel of the step.
+inline void fill_pdl_attribute(cudaLaunchAttribute* attr) {
+  attr->id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr->val.programmaticStreamSerializationAllowed = 1;
 }
 
 }  // namespace fastkv

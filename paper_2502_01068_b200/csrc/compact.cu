@@ -39,6 +39,8 @@ __device__ __forceinline__ int owner_of_slot(const int* cu_k, int k_uniform, int
 }  // namespace
 
 __global__ void __launch_bounds__(kGatherThreads) compact_rows_kernel(const CompactParams p) {
+  pdl_wait();                  // the indices come from the kernel before this one
+  pdl_launch_dependents();
   int ji = 0;
   while (ji + 1 < p.n_jobs && static_cast<int>(blockIdx.x) >= p.job[ji + 1].first_block) ++ji;
   const GatherJob& job = p.job[ji];
@@ -111,8 +113,15 @@ cudaError_t launch_compact(CompactParams& p, cudaStream_t stream) {
     p.job[i].n_blocks = static_cast<int>(want);
     first += static_cast<int>(want);
   }
-  compact_rows_kernel<<<first, kGatherThreads, 0, stream>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(first);
+  cfg.blockDim = dim3(kGatherThreads);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  fill_pdl_attribute(&attr[0]);
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, compact_rows_kernel, static_cast<const CompactParams&>(p));
 }
 
 }  // namespace fastkv

@@ -169,6 +169,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   tc_fence_after_sync();
   const uint32_t tmem_base = bars->tmem_base;
   volatile int* abort_flag = &bars->abort_flag;
+  pdl_launch_dependents();     // the pooling kernel may be brought up; it waits for this grid to finish
 
   if (warp == 0 || warp == 2) {
     // ---------------- TMA producers (warp 0: pipeline 1 from HBM, warp 2: pipeline 2 from L2) ----------------
@@ -454,6 +455,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kPoolThreads) pool_rows_kernel(const PoolRowsParams p) {
   extern __shared__ float sm[];
+  pdl_wait();                  // the un-pooled scores come from the scoring kernel before this one
+  pdl_launch_dependents();
   const int b = blockIdx.y;
   const int row0 = p.cu_seqlens ? p.cu_seqlens[b] : 0;
   const int L = p.cu_seqlens ? p.cu_seqlens[b + 1] - row0 : p.total_len;
@@ -534,9 +537,16 @@ cudaError_t launch_pool_rows(const PoolRowsParams& p, int max_len, int batch, cu
     if (e != cudaSuccess) return e;
     configured = smem;
   }
-  dim3 grid((max_len + kPoolKeys - 1) / kPoolKeys, batch);
-  pool_rows_kernel<<<grid, kPoolThreads, smem, stream>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((max_len + kPoolKeys - 1) / kPoolKeys, batch);
+  cfg.blockDim = dim3(kPoolThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  fill_pdl_attribute(&attr[0]);
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, pool_rows_kernel, p);
 }
 
 }  // namespace fastkv

@@ -52,17 +52,21 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
   constexpr bool CACHED = ITEMS > 0;
   constexpr int R = CACHED ? ITEMS : 1;
   const int rank = static_cast<int>(cluster.block_rank());
-  const int row = blockIdx.y, b = blockIdx.z;
+  const bool second = static_cast<int>(blockIdx.y) >= p.set[0].n_rows;
+  const SelectSet& ps = p.set[second ? 1 : 0];
+  const int row = static_cast<int>(blockIdx.y) - (second ? p.set[0].n_rows : 0), b = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t lt_mask = (1u << lane) - 1u;
 
+  pdl_wait();                  // the scores come from the kernel before this one
+  pdl_launch_dependents();
   const int row0 = p.cu_seqlens ? p.cu_seqlens[b] : 0;
   const int L = p.cu_seqlens ? p.cu_seqlens[b + 1] - row0 : p.total_len;
-  const int out0 = p.cu_k ? p.cu_k[b] : b * p.k_uniform;
-  int k = p.cu_k ? p.cu_k[b + 1] - out0 : p.k_uniform;
+  const int out0 = ps.cu_k ? ps.cu_k[b] : b * ps.k_uniform;
+  int k = ps.cu_k ? ps.cu_k[b + 1] - out0 : ps.k_uniform;
   const int w = p.force_window ? p.window : 0;
-  const float* S = p.scores + static_cast<size_t>(row) * p.ld_scores + row0;
-  int* out = p.idx + static_cast<size_t>(row) * p.ld_idx + out0;
+  const float* S = ps.scores + static_cast<size_t>(row) * ps.ld_scores + row0;
+  int* out = ps.idx + static_cast<size_t>(row) * ps.ld_idx + out0;
 
   // budget outside [w, L]: clamp so that writes stay inside this sequence's output segment,
   // and report it (the whole cluster takes the same branch: k, L, w are uniform)
@@ -241,7 +245,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
 namespace {
 
 template <int CLUSTER, int ITEMS>
-cudaError_t launch_select_t(const SelectParams& p, int n_rows, int batch, cudaStream_t stream) {
+cudaError_t launch_select_t(const SelectParams& p, int batch, cudaStream_t stream) {
   if (CLUSTER > 8) {
     static bool configured = false;
     if (!configured) {
@@ -252,31 +256,32 @@ cudaError_t launch_select_t(const SelectParams& p, int n_rows, int batch, cudaSt
     }
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(CLUSTER, n_rows, batch);
+  cfg.gridDim = dim3(CLUSTER, p.set[0].n_rows + p.set[1].n_rows, batch);
   cfg.blockDim = dim3(kSelThreads);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = CLUSTER;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  fill_pdl_attribute(&attr[1]);
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, select_topk_kernel<CLUSTER, ITEMS>, p);
 }
 
 }  // namespace
 
-cudaError_t launch_select(const SelectParams& p, int n_rows, int batch, int max_len, cudaStream_t stream) {
+cudaError_t launch_select(const SelectParams& p, int batch, int max_len, cudaStream_t stream) {
   // 8-CTA clusters: every problem of a layer (KV heads plus the TSP row) is resident at once on a
   // 148-SM part.  The per-thread register cache is picked from the longest sequence.
   const long long per_cta = (static_cast<long long>(max_len) + 7) / 8;
-  if (per_cta <= 4 * kSelThreads) return launch_select_t<8, 4>(p, n_rows, batch, stream);
-  if (per_cta <= 8 * kSelThreads) return launch_select_t<8, 8>(p, n_rows, batch, stream);
-  if (per_cta <= 16 * kSelThreads) return launch_select_t<8, 16>(p, n_rows, batch, stream);
-  if (per_cta <= 32 * kSelThreads) return launch_select_t<8, 32>(p, n_rows, batch, stream);
-  return launch_select_t<8, 0>(p, n_rows, batch, stream);
+  if (per_cta <= 4 * kSelThreads) return launch_select_t<8, 4>(p, batch, stream);
+  if (per_cta <= 8 * kSelThreads) return launch_select_t<8, 8>(p, batch, stream);
+  if (per_cta <= 16 * kSelThreads) return launch_select_t<8, 16>(p, batch, stream);
+  if (per_cta <= 32 * kSelThreads) return launch_select_t<8, 32>(p, batch, stream);
+  return launch_select_t<8, 0>(p, batch, stream);
 }
 
 }  // namespace fastkv

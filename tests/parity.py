@@ -30,7 +30,7 @@ def host(t: torch.Tensor, dtype) -> np.ndarray:
 
 
 def gpu_layer(wl: W.Workload, x: W.LayerInputs, *, pool_mode=None, agg_order=B.GROUP_THEN_POOL,
-              force_window=True, ragged_api=None, keep_device=False) -> Dict[str, np.ndarray]:
+              force_window=True, ragged_api=None, keep_device=False, fused_select=True) -> Dict[str, np.ndarray]:
     """score -> select_kv -> select_tsp -> compact through the binding.  `ragged_api` forces the
     cu_seqlens / cu_k form of the interface even for a single sequence."""
     lens = np.diff(x.cu_seqlens).tolist()
@@ -60,12 +60,16 @@ def gpu_layer(wl: W.Workload, x: W.LayerInputs, *, pool_mode=None, agg_order=B.G
 
     b_kv, keep1 = budget(wl.k_kv)
     idx_kv = torch.full((wl.n_kv_heads, b_kv.total), -1, dtype=torch.int32, device="cuda")
-    B.fastkv_select_kv(shape, s_kv, b_kv, idx_kv, ws)
     b_tsp = idx_tsp = keep2 = None
     if wl.k_tsp is not None:
         b_tsp, keep2 = budget(wl.k_tsp)
         idx_tsp = torch.full((b_tsp.total,), -1, dtype=torch.int32, device="cuda")
-        B.fastkv_select_tsp(shape, s_tsp, b_tsp, idx_tsp, ws)
+    if fused_select and wl.k_tsp is not None:
+        B.fastkv_select(shape, s_kv, b_kv, idx_kv, s_tsp, b_tsp, idx_tsp, ws)
+    else:
+        B.fastkv_select_kv(shape, s_kv, b_kv, idx_kv, ws)
+        if wl.k_tsp is not None:
+            B.fastkv_select_tsp(shape, s_tsp, b_tsp, idx_tsp, ws)
     k_out = torch.zeros((wl.n_kv_heads, b_kv.total, wl.head_dim), dtype=torch.int16, device="cuda")
     v_out = torch.zeros_like(k_out) if v is not None else None
     hid_out = pos_out = None
