@@ -1,28 +1,37 @@
 // Compaction of the kept K/V rows, hidden states and position ids (Alg. 1: C <- update(K, V);
-// the reduced hidden states x).  Pure byte movement: every row is copied with 16-byte vector
-// loads and stores, several independent loads in flight per thread before the first store.
+// the reduced hidden states x).  Pure byte movement, done with the bulk-copy engine: every warp
+// owns a small ring of 8 KB shared-memory stages; the kept rows of a chunk are pulled in with
+// cp.async.bulk (one copy per row, issued by the lane that resolved the row's index) and, because
+// kept rows are contiguous in the output, pushed out again with a single bulk store per chunk.
+// No data passes through registers; several chunks per warp are in flight at any time.
 #include "compact.cuh"
 
 namespace fastkv {
 
 namespace {
 
-constexpr int kGatherThreads = 256;
-constexpr int kGatherWarps = kGatherThreads / 32;
-constexpr int kUnroll = 4;
+constexpr int kChunkBytes = 8192;
+constexpr int kStages = 4;                 // chunks in flight per warp
+constexpr int kCompactWarps = 6;
+constexpr int kCompactThreads = kCompactWarps * 32;
+constexpr int kCompactSmem = kCompactWarps * kStages * kChunkBytes + 1024;
 
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
-  return v;
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
 }
-__device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
-  asm volatile("st.global.cs.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
-               "r"(v.w)
+__device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(smem_src)),
+               "r"(bytes)
                : "memory");
 }
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // sequence that owns output slot j: the last b with cu_k[b] <= j
 __device__ __forceinline__ int owner_of_slot(const int* cu_k, int k_uniform, int batch, int j) {
@@ -38,84 +47,157 @@ __device__ __forceinline__ int owner_of_slot(const int* cu_k, int k_uniform, int
 
 }  // namespace
 
-__global__ void __launch_bounds__(kGatherThreads) compact_rows_kernel(const CompactParams p) {
+__global__ void __launch_bounds__(kCompactThreads, 1) compact_rows_kernel(const CompactParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
+  __shared__ uint64_t full[kCompactWarps][kStages];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint8_t* const ring = smem + warp * kStages * kChunkBytes;
+  if (lane == 0) {
+    for (int s = 0; s < kStages; ++s) mbar_init(&full[warp][s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) abort_flag = 0;
+  __syncthreads();
   pdl_wait();                  // the indices come from the kernel before this one
   pdl_launch_dependents();
-  int ji = 0;
-  while (ji + 1 < p.n_jobs && static_cast<int>(blockIdx.x) >= p.job[ji + 1].first_block) ++ji;
-  const GatherJob& job = p.job[ji];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int chunks = job.row_chunks;
-  const long long total_rows = static_cast<long long>(job.heads) * job.rows;
-  // a warp copies `rows_per_step` rows at a time: narrow rows share a warp, wide rows loop
-  const int lanes_per_row = chunks >= 32 ? 32 : (chunks > 16 ? 32 : (chunks > 8 ? 16 : (chunks > 4 ? 8 : 4)));
-  const int rows_per_step = 32 / lanes_per_row;
-  const int sub = lane / lanes_per_row, lane_in_row = lane % lanes_per_row;
-  const long long warp_global = static_cast<long long>(blockIdx.x - job.first_block) * kGatherWarps + warp;
-  const long long warp_count = static_cast<long long>(job.n_blocks) * kGatherWarps;
 
-  for (long long r0 = warp_global * rows_per_step; r0 < total_rows; r0 += warp_count * rows_per_step) {
-    const long long r = r0 + sub;
-    if (r >= total_rows) continue;
-    const int head = static_cast<int>(r / job.rows);
-    const int j = static_cast<int>(r - static_cast<long long>(head) * job.rows);
-    const int b = owner_of_slot(job.cu_k, job.k_uniform, p.batch, j);
-    const int row0 = p.cu_seqlens ? p.cu_seqlens[b] : 0;
-    const int L = p.cu_seqlens ? p.cu_seqlens[b + 1] - row0 : p.total_len;
-    const int i = job.idx[static_cast<long long>(head) * job.ld_idx + j];
-    if (i < 0 || i >= L) {           // never read outside the sequence: skip the row and report it
-      if (lane_in_row == 0) raise_status(p.hdr, FASTKV_ERR_DEVICE_INDEX, SITE_COMPACT_INDEX);
-      continue;
+  const long long gw = static_cast<long long>(blockIdx.x) * kCompactWarps + warp;
+  const long long n_warps = static_cast<long long>(gridDim.x) * kCompactWarps;
+  const long long my_chunks = gw < p.total_chunks ? (p.total_chunks - gw + n_warps - 1) / n_warps : 0;
+
+  // Issue the loads of this warp's c-th chunk into stage c % kStages (warp-collective); returns what
+  // lane 0 needs to store the chunk later.
+  struct Pending { uint8_t* dst; uint32_t bytes; uint32_t valid; uint32_t row_bytes; };
+  auto issue = [&](long long c) -> Pending {
+    const long long chunk = gw + c * n_warps;
+    int ji = 0;
+    while (ji + 1 < p.n_jobs && chunk >= p.job[ji + 1].first_chunk) ++ji;
+    const GatherJob& job = p.job[ji];
+    const long long lc = chunk - job.first_chunk;
+    const int s = static_cast<int>(c % kStages);
+    uint8_t* const stage = ring + s * kChunkBytes;
+    const long long row_bytes = static_cast<long long>(job.row_chunks) * 16;
+    long long r;                       // output row of this lane
+    uint32_t bytes, src_off = 0;       // bytes this lane copies, offset inside the source row
+    bool active;
+    if (job.pieces_per_row > 1) {      // long rows: one piece of one row per chunk, lane 0 copies it
+      r = lc / job.pieces_per_row;
+      src_off = static_cast<uint32_t>(lc - r * job.pieces_per_row) * kChunkBytes;
+      bytes = static_cast<uint32_t>(min(static_cast<long long>(kChunkBytes), row_bytes - src_off));
+      active = lane == 0;
+    } else {                           // short rows: up to 32 rows per chunk, one per lane
+      r = lc * job.rows_per_chunk + lane;
+      bytes = static_cast<uint32_t>(row_bytes);
+      active = lane < job.rows_per_chunk && r < static_cast<long long>(job.heads) * job.rows;
     }
-    const long long tok = static_cast<long long>(row0) + i;
-    const uint4* src = reinterpret_cast<const uint4*>(job.src + tok * job.src_tok_bytes +
-                                                      head * job.src_head_bytes);
-    uint4* dst = reinterpret_cast<uint4*>(job.dst) + r * chunks;
-    if (job.src != nullptr) {
-      for (int c0 = lane_in_row; c0 < chunks; c0 += lanes_per_row * kUnroll) {
-        uint4 v[kUnroll];
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u)
-          if (c0 + u * lanes_per_row < chunks) v[u] = ld_stream(src + c0 + u * lanes_per_row);
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u)
-          if (c0 + u * lanes_per_row < chunks) st_stream(dst + c0 + u * lanes_per_row, v[u]);
+    const uint8_t* src = nullptr;
+    bool valid = false;
+    if (active) {
+      const int head = static_cast<int>(r / job.rows);
+      const int j = static_cast<int>(r - static_cast<long long>(head) * job.rows);
+      const int b = owner_of_slot(job.cu_k, job.k_uniform, p.batch, j);
+      const int row0 = p.cu_seqlens ? p.cu_seqlens[b] : 0;
+      const int L = p.cu_seqlens ? p.cu_seqlens[b + 1] - row0 : p.total_len;
+      const int i = job.idx[static_cast<long long>(head) * job.ld_idx + j];
+      if (i < 0 || i >= L) {           // never read outside the sequence: skip the row and report it
+        raise_status(p.hdr, FASTKV_ERR_DEVICE_INDEX, SITE_COMPACT_INDEX);
+      } else {
+        valid = true;
+        const long long tok = static_cast<long long>(row0) + i;
+        src = job.src + tok * job.src_tok_bytes + head * job.src_head_bytes + src_off;
+        if (job.pos_src != nullptr && head == 0 && src_off == 0) job.pos_dst[j] = job.pos_src[tok];
       }
     }
-    if (job.pos_src != nullptr && head == 0 && lane_in_row == 0) job.pos_dst[j] = job.pos_src[tok];
+    const uint32_t vmask = __ballot_sync(0xffffffffu, valid && job.src != nullptr);
+    const uint32_t amask = __ballot_sync(0xffffffffu, active);
+    const uint32_t bytes0 = __shfl_sync(0xffffffffu, bytes, 0);          // every row of a chunk has this size
+    const long long r_first = __shfl_sync(0xffffffffu, r, 0);
+    const uint32_t off_first = __shfl_sync(0xffffffffu, src_off, 0);
+    Pending pend;
+    pend.valid = vmask;
+    pend.row_bytes = bytes0;
+    pend.dst = job.dst + r_first * row_bytes + off_first;
+    pend.bytes = (vmask == amask) ? static_cast<uint32_t>(__popc(amask)) * bytes0 : 0u;   // 0: store row by row
+    // one phase of the stage's barrier per chunk, even when nothing is loaded
+    if (lane == 0) mbar_arrive_expect_tx(&full[warp][s], static_cast<uint32_t>(__popc(vmask)) * bytes0);
+    __syncwarp();
+    if (valid && job.src != nullptr)
+      bulk_load(stage + (job.pieces_per_row > 1 ? 0u : lane * bytes0), src, bytes0, &full[warp][s]);
+    return pend;
+  };
+
+  Pending pending[kStages];
+  constexpr int kAhead = kStages - 2;      // loads in flight per warp; one more stage is being stored
+  const long long prologue = my_chunks < kAhead ? my_chunks : kAhead;
+  for (long long c = 0; c < prologue; ++c) pending[c % kStages] = issue(c);
+  for (long long c = 0; c < my_chunks; ++c) {
+    const long long ahead = c + kAhead;
+    if (ahead < my_chunks) {
+      // that stage was stored two chunks ago: all but the latest store must have read their stage
+      if (lane == 0) bulk_wait_read<1>();
+      __syncwarp();
+      pending[ahead % kStages] = issue(ahead);
+    }
+    const int s = static_cast<int>(c % kStages);
+    const Pending pend = pending[s];
+    if (lane == 0) {
+      const bool ok = mbar_wait_bounded(&full[warp][s], static_cast<uint32_t>((c / kStages) & 1), &abort_flag, p.hdr,
+                                        SITE_COMPACT_WAIT);
+      if (ok && pend.valid != 0) {
+        uint8_t* const stage = ring + s * kChunkBytes;
+        if (pend.bytes != 0) {
+          bulk_store(pend.dst, stage, pend.bytes);      // every row of the chunk is there: one store
+        } else {
+          for (int i = 0; i < 32; ++i)                    // some row was skipped: store the others one by one
+            if ((pend.valid >> i) & 1u) bulk_store(pend.dst + i * pend.row_bytes, stage + i * pend.row_bytes, pend.row_bytes);
+        }
+      }
+      bulk_commit();
+    }
+    __syncwarp();
   }
+  if (lane == 0) bulk_wait_all();
 }
 
 cudaError_t launch_compact(CompactParams& p, cudaStream_t stream) {
-  // blocks are shared out among the jobs in proportion to the bytes they move
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) {
     int v = 0;
     if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
   }
-  const int budget = sms * 8;
-  double bytes[3] = {0, 0, 0}, total = 0;
+  long long first = 0;
   for (int i = 0; i < p.n_jobs; ++i) {
-    bytes[i] = static_cast<double>(p.job[i].heads) * p.job[i].rows * (p.job[i].row_chunks * 16.0 + 4.0);
-    total += bytes[i];
+    GatherJob& j = p.job[i];
+    const long long row_bytes = static_cast<long long>(j.row_chunks) * 16;
+    const long long rows = static_cast<long long>(j.heads) * j.rows;
+    if (row_bytes > kChunkBytes) {
+      j.pieces_per_row = static_cast<int>((row_bytes + kChunkBytes - 1) / kChunkBytes);
+      j.rows_per_chunk = 1;
+    } else {
+      j.pieces_per_row = 1;
+      long long rpc = row_bytes > 0 ? kChunkBytes / row_bytes : 32;
+      j.rows_per_chunk = static_cast<int>(rpc > 32 ? 32 : (rpc < 1 ? 1 : rpc));
+    }
+    j.first_chunk = first;
+    first += j.pieces_per_row > 1 ? rows * j.pieces_per_row : (rows + j.rows_per_chunk - 1) / j.rows_per_chunk;
   }
-  if (total <= 0) return cudaSuccess;
-  int first = 0;
-  for (int i = 0; i < p.n_jobs; ++i) {
-    const GatherJob& j = p.job[i];
-    const int lanes_per_row = j.row_chunks >= 32 ? 32 : (j.row_chunks > 16 ? 32 : (j.row_chunks > 8 ? 16 : (j.row_chunks > 4 ? 8 : 4)));
-    const long long steps = (static_cast<long long>(j.heads) * j.rows * lanes_per_row + 31) / 32;
-    long long want = static_cast<long long>(budget * (bytes[i] / total) + 0.999);
-    const long long cap = (steps + kGatherWarps - 1) / kGatherWarps;
-    if (want > cap) want = cap;
-    if (want < 1) want = 1;
-    p.job[i].first_block = first;
-    p.job[i].n_blocks = static_cast<int>(want);
-    first += static_cast<int>(want);
+  p.total_chunks = first;
+  if (first == 0) return cudaSuccess;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(compact_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCompactSmem);
+    if (e != cudaSuccess) return e;
+    configured = true;
   }
+  long long blocks = (first + kCompactWarps - 1) / kCompactWarps;
+  if (blocks > sms) blocks = sms;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(first);
-  cfg.blockDim = dim3(kGatherThreads);
+  cfg.gridDim = dim3(static_cast<unsigned>(blocks));
+  cfg.blockDim = dim3(kCompactThreads);
+  cfg.dynamicSmemBytes = kCompactSmem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   fill_pdl_attribute(&attr[0]);

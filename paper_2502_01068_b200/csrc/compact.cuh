@@ -20,13 +20,15 @@ struct GatherJob {
   int k_uniform;
   const int* pos_src;         // optional int32 side channel gathered with head 0 rows
   int* pos_dst;
-  int first_block;            // blocks [first_block, first_block + n_blocks) work on this job
-  int n_blocks;
+  int rows_per_chunk;         // rows copied per 8 KB chunk (short rows), or 1
+  int pieces_per_row;         // chunks per row (rows longer than a chunk), or 1
+  long long first_chunk;      // chunks [first_chunk, next job's first_chunk) belong to this job
 };
 
 struct CompactParams {
   GatherJob job[3];
   int n_jobs;
+  long long total_chunks;
   int batch;
   int total_len;
   const int* cu_seqlens;
