@@ -78,6 +78,22 @@ def measured_peaks() -> dict:
     return {"hbm_gbs": 6650.0, "source": "fallback (earlier measurement on this pool)"}
 
 
+def profiled_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch of `kernel` from the committed ncu summary of this workload, or None."""
+    tag = {"llama8b_128k_tsp_layer": "llama8b_128k"}.get(workload)
+    if tag is None:
+        return None
+    path = os.path.join(ROOT, "profiles", "%s_%s.txt" % (kernel, tag))
+    try:
+        with open(path) as f:
+            for line in f:
+                if line.startswith("dram_bytes_per_launch:"):
+                    return int(line.split(":")[1])
+    except OSError:
+        pass
+    return None
+
+
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
 
@@ -128,6 +144,22 @@ class ClockSampler(threading.Thread):
             self.join(timeout=2.0)
         return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """The slowest rank's time: every multi-GPU number is the max over ranks (device-timed per rank)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_throughput(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Weak scaling over independent layers: all ranks' tokens over the slowest rank's step time."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
 
 
 def oracle_baseline(wl: W.Workload, x: W.LayerInputs, budget_s: float = 20.0, max_reps: int = 3) -> dict:
@@ -286,13 +318,9 @@ def main() -> None:
     launches = B.fastkv_kernel_launches() - launches0
     total_ms = ev[0][0].elapsed_time(ev[-1][4])
     call_ms = [statistics.mean(ev[i][c].elapsed_time(ev[i][c + 1]) for i in range(steps)) for c in range(4)]
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, "cuda")
     ms_per_step = total_ms / steps
-    value = world * total / (ms_per_step * 1e-3)
+    value = whole_job_throughput(total, world, ms_per_step)
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies timed) -------------
     e2e = None
@@ -324,11 +352,7 @@ def main() -> None:
         for _ in range(args.e2e_steps):
             host_step()                                   # synchronises: outputs are on the host
         e2e_s = (time.perf_counter() - t0) / args.e2e_steps
-        if world > 1:
-            import torch.distributed as dist
-            t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = max_over_ranks(e2e_s, world, "cuda")
         h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hh, hp))
         d2h = sum(t.numel() * t.element_size() for t in (o_idx_kv, o_idx_tsp, o_k, o_v, o_h, o_p))
         e2e = {"value": world * total / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -356,7 +380,8 @@ def main() -> None:
         "e2e": e2e,
         "roofline": {"bound": "hbm", "kernel": "compact_rows_kernel", "achieved": compact_gbs,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": compact_gbs / peaks["hbm_gbs"],
-                     "peak_source": peaks["source"], "algorithmic_bytes": ab["compact"], "traffic": None,
+                     "peak_source": peaks["source"], "algorithmic_bytes": ab["compact"],
+                     "traffic": profiled_traffic("compact_rows_kernel", args.workload),
                      "ms": call_ms[3]},
         "step_roofline": {"bytes_rw": ab["step_rw"], "bytes_rows_once": ab["step_min"], "achieved_gbs": step_gbs,
                           "frac_of_measured": step_gbs / peaks["hbm_gbs"],
