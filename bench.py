@@ -162,7 +162,7 @@ def whole_job_throughput(tokens_per_rank: int, world: int, ms_per_step: float) -
     return world * tokens_per_rank / (ms_per_step * 1e-3)
 
 
-def oracle_baseline(wl: W.Workload, x: W.LayerInputs, budget_s: float = 20.0, max_reps: int = 3) -> dict:
+def oracle_baseline(wl: W.Workload, x: W.LayerInputs, budget_s: float = 15.0, max_reps: int = 16) -> dict:
     """Times the fp64 oracle, as it stands, on this machine's host cores on the same layer."""
     import oracle
     from oracle.layer import layer_step
