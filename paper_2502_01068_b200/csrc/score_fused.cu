@@ -466,11 +466,16 @@ __global__ void __launch_bounds__(kPoolThreads) pool_rows_kernel(const PoolRowsP
   const int span = kPoolKeys + 2 * r;
   const int sub = p.per_head ? p.group : 1;
   const int rows = p.n_kv_heads * sub;
-  for (int item = threadIdx.x; item < rows * span; item += blockDim.x) {
-    const int row = item / span, o = item - row * span;
+  // each thread fetches its position(s) for every row; eight rows' loads are in flight together
+  for (int o = threadIdx.x; o < span; o += blockDim.x) {
     const int key = k0 - r + o;
-    const float* src = p.a + static_cast<size_t>(row) * p.ld_a + row0 + key;
-    sm[item] = (key >= 0 && key < L) ? __ldg(src) + __ldg(src + p.plane_stride) : 0.0f;
+    const bool inside = key >= 0 && key < L;
+    const float* src = p.a + row0 + key;
+#pragma unroll 8
+    for (int row = 0; row < rows; ++row) {
+      const float* s0 = src + static_cast<size_t>(row) * p.ld_a;
+      sm[row * span + o] = inside ? __ldg(s0) + __ldg(s0 + p.plane_stride) : 0.0f;
+    }
   }
   __syncthreads();
   const float inv_p = 1.0f / static_cast<float>(p.pool_kernel);
