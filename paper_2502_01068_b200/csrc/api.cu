@@ -86,7 +86,7 @@ Layout make_layout(const fastkv_shape& s) {
   l.f_off_partial = off;
   off += round_up(sizeof(float2) * static_cast<size_t>(phases) * kFusedMaxCtas * l.npad, 256);
   l.f_off_a = off;
-  off += 2 * round_up(sizeof(float) * static_cast<size_t>(l.f_rows) * l.ld_logits, 256);   // two planes
+  off += round_up(sizeof(float) * static_cast<size_t>(l.f_rows) * l.ld_logits, 256);
   l.f_bytes = off;
   if (l.f_bytes > l.bytes) l.bytes = l.f_bytes;     // one size serves whichever path runs
   return l;
@@ -281,7 +281,6 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
     fp.per_head = s.agg_order == FASTKV_POOL_THEN_GROUP;
     fp.scale_log2 = scale_log2; fp.cu_seqlens = s.cu_seqlens;
     fp.a_out = reinterpret_cast<float*>(ws + lay.f_off_a); fp.ld_a = lay.ld_logits;
-    fp.plane_stride = static_cast<long long>(round_up(sizeof(float) * static_cast<size_t>(lay.f_rows) * lay.ld_logits, 256) / sizeof(float));
     const char* lead = std::getenv("FASTKV_FUSED_LEAD");     // tuning knob: phases of K kept in flight in L2
     fp.max_lead = lead ? std::atoi(lead) : 3;
     if (fp.max_lead < 1) fp.max_lead = 1;
@@ -294,7 +293,7 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
     PoolRowsParams rp;
     rp.total_len = s.total_len; rp.n_kv_heads = s.n_kv_heads; rp.group = G; rp.window = s.window;
     rp.per_head = fp.per_head; rp.pool_kernel = s.pool_kernel; rp.pool_mode = s.pool_mode;
-    rp.cu_seqlens = s.cu_seqlens; rp.a = fp.a_out; rp.ld_a = lay.ld_logits; rp.plane_stride = fp.plane_stride;
+    rp.cu_seqlens = s.cu_seqlens; rp.a = fp.a_out; rp.ld_a = lay.ld_logits;
     rp.scores_kv = scores_kv; rp.ld_scores = s.total_len; rp.scores_tsp = scores_tsp;
     if (sizeof(float) * static_cast<size_t>(lay.f_rows) * (kPoolKeys + s.pool_kernel) > 200 * 1024)
       return fail(FASTKV_ERR_UNSUPPORTED, "heads x pool halo do not fit the pooling kernel's shared memory");

@@ -45,9 +45,8 @@ struct FusedParams {
   float scale_log2;
   const int* cu_seqlens;
   int max_lead;               // phases the HBM pipeline may run ahead of the re-read pipeline
-  float* a_out;               // [2][Hkv or Hq][ld_a] un-pooled scores, one plane per accumulator-column half
+  float* a_out;               // [Hkv or Hq][ld_a] un-pooled scores
   long long ld_a;
-  long long plane_stride;     // elements between the two planes
   float2* partial;            // [phases][CTAs][NPAD]
   int* counters;              // [phases] CTAs that published their statistics (zero before launch)
   WorkspaceHeader* hdr;
@@ -57,9 +56,8 @@ struct PoolRowsParams {
   int total_len, n_kv_heads, group, window, per_head;
   int pool_kernel, pool_mode;
   const int* cu_seqlens;
-  const float* a;             // two planes, plane_stride apart; their sum is the un-pooled score
+  const float* a;             // [Hkv or Hq][ld_a] un-pooled scores
   long long ld_a;
-  long long plane_stride;
   float* scores_kv;
   long long ld_scores;
   float* scores_tsp;

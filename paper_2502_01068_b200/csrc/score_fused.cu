@@ -77,7 +77,6 @@ __device__ __forceinline__ bool wait_smem_counter(volatile int* flag, int target
   const long long t0 = clock64();
   unsigned spins = 0;
   while (*flag < target) {
-    __nanosleep(64);
     if ((++spins & 0x3Fu) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) {
       *abort_flag = 1;
       raise_status(hdr, FASTKV_ERR_DEVICE_TIMEOUT, site);
@@ -150,7 +149,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     }
     for (int i = 0; i < kAcc; ++i) {
       mbar_init(&bars->acc1_full[i], 1); mbar_init(&bars->acc1_empty[i], kGroupWarps);   // every warp of the group
-      mbar_init(&bars->acc2_full[i], 1); mbar_init(&bars->acc2_empty[i], kGroupWarps);
+      mbar_init(&bars->acc2_full[i], 1); mbar_init(&bars->acc2_empty[i], 4);             // the four warps of one set
     }
     bars->abort_flag = 0;
     bars->p1_done = 0;
@@ -334,15 +333,15 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     }
   } else {
     // ---------------- group B: pass 2, normalise and sum over window rows / group ----------------
-    // Same (quarter, half) split as group A; each half writes its partial sums to its own plane of
-    // a_out, and the pooling kernel adds the two planes.
+    // Two sets of four warps (one per tensor-memory lane quarter) take alternate tiles, so two tiles
+    // are in flight and one set's waits and stores overlap the other set's exponentials.  A warp
+    // handles all query rows of its 32 keys; the normaliser is read from shared memory (broadcast).
     const int gw = warp - kCtrlWarps - kGroupWarps;
-    const int quarter = warp & 3, half = gw >> 2;
+    const int quarter = warp & 3, set = gw >> 2;
     const int key_in_tile = quarter * 32 + lane;
     const int bt = threadIdx.x - (kCtrlWarps + kGroupWarps) * 32;   // 0..255 within the group
     const int n_rows = p.n_rows, G = p.group;
-    const int col0 = half * CPW;
-    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + kAcc * NPAD + col0;
+    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + kAcc * NPAD;
     constexpr int kParts = kGroupWarps * 32 / NPAD;
     int it = 0, u = 0;
     bool ok = true;
@@ -374,14 +373,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         float mm = -INFINITY, ll = 0.0f;
 #pragma unroll
         for (int q = 0; q < kParts; ++q) merge_stats(mm, ll, merge_buf[q * NPAD + bt].x, merge_buf[q * NPAD + bt].y);
-        norm[bt] = (bt < n_rows && ll > 0.0f) ? make_float2(mm, 1.0f / ll) : make_float2(0.0f, 0.0f);
+        // (-row max, 1 / row sum); rows beyond G * w contribute nothing
+        norm[bt] = (bt < n_rows && ll > 0.0f) ? make_float2(-mm, 1.0f / ll) : make_float2(0.0f, 0.0f);
       }
       group_sync<2>();
-      float nm[CPW], nil[CPW];                           // -(row max) and 1 / (row sum) of this warp's rows
-#pragma unroll
-      for (int n = 0; n < CPW; ++n) { const float2 st = norm[col0 + n]; nm[n] = -st.x; nil[n] = st.y; }
       const int win_start = w.L - p.window;
       for (int i = 0; i < w.n; ++i, ++it) {
+        if ((it & 1) != set) continue;                   // the other set's tile
         const int a = it % kAcc;
         ok = mbar_wait_bounded(&bars->acc2_full[a], (it / kAcc) & 1, abort_flag, p.hdr, SITE_FUSED_ACC_FULL);
         ok = __all_sync(0xffffffffu, ok);
@@ -394,22 +392,24 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
         for (int q = 0; q < 8; ++q) a_h[q] = 0.0f;
 #pragma unroll
-        for (int c = 0; c < CPW / 16; ++c) {
+        for (int c = 0; c < NPAD / 16; ++c) {
           float pr[16];
           tmem_ld_32x16(lane_base + a * NPAD + c * 16, pr);
-          if (c == CPW / 16 - 1) {                       // this warp's part of the accumulator is in registers
+          if (c == NPAD / 16 - 1) {                      // the accumulator is in registers: hand it back
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->acc2_empty[a]);
           }
-          const int n_valid = n_rows - col0 - c * 16;
+          const int n_valid = n_rows - c * 16;
 #pragma unroll
-          for (int x = 0; x < 16; ++x)
-            pr[x] = (x < n_valid) ? ex2(fmaf(pr[x], p.scale_log2, nm[c * 16 + x])) * nil[c * 16 + x] : 0.0f;
+          for (int x = 0; x < 16; ++x) {
+            const float2 st = norm[c * 16 + x];
+            pr[x] = (x < n_valid) ? ex2(fmaf(pr[x], p.scale_log2, st.x)) * st.y : 0.0f;
+          }
           if (!tile_unmasked) {                          // causal: key i <= t_j, j = n / G
 #pragma unroll
             for (int x = 0; x < 16; ++x)
-              if (x < n_valid && key > win_start + (col0 + c * 16 + x) / G) pr[x] = 0.0f;
+              if (x < n_valid && key > win_start + (c * 16 + x) / G) pr[x] = 0.0f;
           }
           if (!p.per_head) {
 #pragma unroll
@@ -423,15 +423,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             }
           }
         }
-        // each column half writes its own plane of partial sums; the pooling kernel adds the two
         if (key < w.L) {
-          float* const plane = p.a_out + static_cast<size_t>(half) * p.plane_stride;
           if (p.per_head) {
 #pragma unroll
             for (int q = 0; q < 8; ++q)
-              if (q < G) plane[static_cast<size_t>(w.g * G + q) * p.ld_a + w.row0 + key] = a_h[q];
+              if (q < G) p.a_out[static_cast<size_t>(w.g * G + q) * p.ld_a + w.row0 + key] = a_h[q];
           } else {
-            plane[static_cast<size_t>(w.g) * p.ld_a + w.row0 + key] = a_g;
+            p.a_out[static_cast<size_t>(w.g) * p.ld_a + w.row0 + key] = a_g;
           }
         }
       }
@@ -474,7 +472,7 @@ __global__ void __launch_bounds__(kPoolThreads) pool_rows_kernel(const PoolRowsP
 #pragma unroll 8
     for (int row = 0; row < rows; ++row) {
       const float* s0 = src + static_cast<size_t>(row) * p.ld_a;
-      sm[row * span + o] = inside ? __ldg(s0) + __ldg(s0 + p.plane_stride) : 0.0f;
+      sm[row * span + o] = inside ? __ldg(s0) : 0.0f;
     }
   }
   __syncthreads();
