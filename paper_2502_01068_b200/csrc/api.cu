@@ -41,7 +41,7 @@ struct Layout {
   // single-pass path (score_fused.cu): same header, its own carving of the rest
   bool fused_shape_ok;        // the shape fits the tensor-memory-resident design on a full B200
   int f_rows;                 // un-pooled rows written by pass 2 (KV heads or query heads)
-  size_t f_off_counters, f_off_flags, f_off_final, f_off_partial, f_off_a, f_zero_bytes, f_bytes;
+  size_t f_off_counters, f_off_partial, f_off_a, f_zero_bytes, f_bytes;
 };
 
 constexpr int kFusedMaxCtas = 148;      // SMs of a B200: one persistent CTA each
@@ -78,11 +78,7 @@ Layout make_layout(const fastkv_shape& s) {
   off = sizeof(WorkspaceHeader);
   l.f_off_counters = off;
   off += round_up(sizeof(int) * phases, 256);
-  l.f_off_flags = off;
-  off += round_up(sizeof(int) * phases, 256);
-  l.f_zero_bytes = off;
-  l.f_off_final = off;
-  off += round_up(sizeof(float2) * static_cast<size_t>(phases) * l.npad, 256);
+  l.f_zero_bytes = off;                     // header + per-phase counters are cleared by fastkv_score
   l.f_off_partial = off;
   off += round_up(sizeof(float2) * static_cast<size_t>(phases) * kFusedMaxCtas * l.npad, 256);
   l.f_off_a = off;
