@@ -41,10 +41,10 @@ struct alignas(16) SelShared {
 
 }  // namespace
 
-// ITEMS > 0: every thread keeps its ITEMS candidates (converted once) in registers for all
-// passes; candidate (warp w, round r, lane l) of a CTA is c_begin + (w * ITEMS + r) * 32 + l, so
-// loads are coalesced and index order is (warp, round, lane).  ITEMS == 0: any chunk size, every
-// pass re-reads the scores (they are L2 resident).
+// Every thread owns `per` consecutive candidates of its CTA's chunk, so index order is thread order
+// and the ordered compaction at the end needs no warp votes, only one scan of per-thread counts.
+// ITEMS > 0: per = ITEMS and the candidates (converted once) stay in registers for all passes.
+// ITEMS == 0: any chunk size; every pass re-reads the scores (they are L2 resident).
 template <int CLUSTER, int ITEMS>
 __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const SelectParams p) {
   cg::cluster_group cluster = cg::this_cluster();
@@ -56,7 +56,6 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
   const SelectSet& ps = p.set[second ? 1 : 0];
   const int row = static_cast<int>(blockIdx.y) - (second ? p.set[0].n_rows : 0), b = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint32_t lt_mask = (1u << lane) - 1u;
 
   pdl_wait();                  // the scores come from the kernel before this one
   pdl_launch_dependents();
@@ -77,19 +76,28 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
   }
   const int n_cand = L - w;          // ranked positions: [0, n_cand)
   const int k_sel = k - w;           // how many of them are kept
-  // contiguous chunk per CTA, contiguous segment of `rounds` 32-wide rounds per warp
-  const int chunk = (n_cand + CLUSTER - 1) / CLUSTER;
+  // contiguous chunk per CTA, `per` consecutive candidates per thread
+  const int chunk = ((n_cand + CLUSTER - 1) / CLUSTER + 3) & ~3;   // multiple of 4: keeps 16-byte alignment
   const int c_begin = min(n_cand, rank * chunk), c_end = min(n_cand, c_begin + chunk);
-  const int rounds = CACHED ? ITEMS : (chunk + kSelThreads - 1) / kSelThreads;
-  const int w_begin = c_begin + warp * rounds * 32;     // may lie beyond c_end (idle warp)
+  const int per = CACHED ? ITEMS : (chunk + kSelThreads - 1) / kSelThreads;
+  const int t_begin = min(c_end, c_begin + tid * per), t_end = min(c_end, t_begin + per);
+  const int n_mine = t_end - t_begin;
 
   uint32_t key[R];
+  uint32_t live = 0;                 // bit r: candidate r exists and still matches the threshold's prefix
   if (CACHED) {
+    const float* mine = S + t_begin;
+    if (n_mine == R && R % 4 == 0 && (reinterpret_cast<uintptr_t>(mine) & 15u) == 0) {
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-      const int i = w_begin + r * 32 + lane;
-      key[r] = (i < c_end) ? order_key(__ldg(S + i)) : 0u;
+      for (int r = 0; r < R; r += 4) {                 // 16-byte loads: a thread's candidates are contiguous
+        const float4 v = __ldg(reinterpret_cast<const float4*>(mine + r));
+        key[r] = order_key(v.x); key[r + 1] = order_key(v.y); key[r + 2] = order_key(v.z); key[r + 3] = order_key(v.w);
+      }
+    } else {
+#pragma unroll
+      for (int r = 0; r < R; ++r) key[r] = (r < n_mine) ? order_key(__ldg(mine + r)) : 0u;
     }
+    live = n_mine >= 32 ? 0xffffffffu : ((1u << n_mine) - 1u);
   }
 
   uint32_t prefix = 0;
@@ -100,16 +108,13 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
       if (CACHED) {
+        if (live != 0) {               // after two passes almost nobody is left
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-          const uint32_t u = key[r];
-          const bool match = (w_begin + r * 32 + lane < c_end) &&
-                             ((pass == 0) || ((u ^ prefix) >> (shift + 8)) == 0);
-          if (match) atomicAdd(&sh.hist[((u >> shift) & 0xFFu) * 32 + lane], 1);
+          for (int r = 0; r < R; ++r)
+            if ((live >> r) & 1u) atomicAdd(&sh.hist[((key[r] >> shift) & 0xFFu) * 32 + lane], 1);
         }
       } else {
-#pragma unroll 4
-        for (int i = c_begin + tid; i < c_end; i += kSelThreads) {
+        for (int i = t_begin; i < t_end; ++i) {
           const uint32_t u = order_key(__ldg(S + i));
           const bool match = (pass == 0) || ((u ^ prefix) >> (shift + 8)) == 0;
           if (match) atomicAdd(&sh.hist[((u >> shift) & 0xFFu) * 32 + lane], 1);
@@ -119,16 +124,16 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
       {
         // 4 threads per bin, each sums (and clears for the next pass) 8 lane counters
         const int bin = tid >> 2, part = tid & 3;
-        int s = 0;
+        int sum = 0;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           int* c = &sh.hist[bin * 32 + ((part * 8 + i + bin) & 31)];
-          s += *c;
+          sum += *c;
           *c = 0;
         }
-        s += __shfl_xor_sync(0xffffffffu, s, 1);
-        s += __shfl_xor_sync(0xffffffffu, s, 2);
-        if (part == 0) sh.block_hist[pass & 1][bin] = s;
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        if (part == 0) sh.block_hist[pass & 1][bin] = sum;
       }
       cluster.sync();
       if (tid < kBins) {               // one bin per thread: sum it over the cluster (DSMEM reads)
@@ -166,30 +171,48 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
         }
       }
       __syncthreads();
-      prefix |= static_cast<uint32_t>(sh.digit) << shift;
+      const uint32_t digit = static_cast<uint32_t>(sh.digit);
+      prefix |= digit << shift;
       k_rem = sh.k_rem;
+      if (CACHED && live != 0) {       // keep only the candidates that share the threshold's digit
+        uint32_t still = 0;
+#pragma unroll
+        for (int r = 0; r < R; ++r) still |= (((key[r] >> shift) & 0xFFu) == digit ? 1u : 0u) << r;
+        live &= still;
+      }
     }
   }
   // prefix = image of the threshold score tau; k_rem = how many candidates equal to tau are kept
   const uint32_t tau = prefix;
   const int need_eq = (k_sel > 0) ? k_rem : 0;
 
-  // counting sweep: candidates above / equal to tau in this warp's segment (warp-uniform counts)
+  // this thread's candidates above / equal to tau
   int n_gt = 0, n_eq = 0;
   if (k_sel > 0) {
+    if (CACHED) {
 #pragma unroll
-    for (int r = 0; r < (CACHED ? R : 1); ++r) {
-      for (int rr = (CACHED ? r : 0); rr < (CACHED ? r + 1 : rounds); ++rr) {
-        const int i = w_begin + rr * 32 + lane;
-        const uint32_t u = CACHED ? key[r] : ((i < c_end) ? order_key(__ldg(S + i)) : 0u);
-        n_gt += __popc(__ballot_sync(0xffffffffu, i < c_end && u > tau));
-        n_eq += __popc(__ballot_sync(0xffffffffu, i < c_end && u == tau));
+      for (int r = 0; r < R; ++r) {
+        n_gt += (r < n_mine && key[r] > tau) ? 1 : 0;
+        n_eq += (r < n_mine && key[r] == tau) ? 1 : 0;
+      }
+    } else {
+      for (int i = t_begin; i < t_end; ++i) {
+        const uint32_t u = order_key(__ldg(S + i));
+        n_gt += (u > tau) ? 1 : 0;
+        n_eq += (u == tau) ? 1 : 0;
       }
     }
   }
-  if (lane == 0) { sh.warp_tot[0][warp] = n_gt; sh.warp_tot[1][warp] = n_eq; }
+  // exclusive scans in thread order: within the warp, then over the 32 warps
+  int gt_incl = n_gt, eq_incl = n_eq;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int va = __shfl_up_sync(0xffffffffu, gt_incl, o), ve = __shfl_up_sync(0xffffffffu, eq_incl, o);
+    if (lane >= o) { gt_incl += va; eq_incl += ve; }
+  }
+  if (lane == 31) { sh.warp_tot[0][warp] = gt_incl; sh.warp_tot[1][warp] = eq_incl; }
   __syncthreads();
-  if (warp == 0) {                   // exclusive scan over the 32 warps
+  if (warp == 0) {
     int a = sh.warp_tot[0][lane], e = sh.warp_tot[1][lane];
     const int a0 = a, e0 = e;
 #pragma unroll
@@ -202,7 +225,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
     if (lane == 31) { sh.counts[0] = a; sh.counts[1] = e; }
   }
   __syncthreads();
-  const int gt_excl = sh.warp_tot[0][warp], eq_excl = sh.warp_tot[1][warp];
+  const int gt_excl = sh.warp_tot[0][warp] + gt_incl - n_gt, eq_excl = sh.warp_tot[1][warp] + eq_incl - n_eq;
   cluster.sync();
   // candidates kept by lower-ranked CTAs (they hold lower indices)
   int g_r[CLUSTER], e_r[CLUSTER];
@@ -220,21 +243,25 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
       eq_before += e_r[r];
     }
   }
-  if (k_sel > 0) {
-    int eq_run = eq_before + eq_excl;                        // rank of the segment's first tau-valued candidate
-    int pos = kept_before + gt_excl + min(eq_run, need_eq) - min(eq_before, need_eq);
+  if (k_sel > 0 && n_gt + n_eq > 0) {
+    int eq_rank = eq_before + eq_excl;                       // rank of this thread's first tau-valued candidate
+    int pos = kept_before + gt_excl + min(eq_rank, need_eq) - min(eq_before, need_eq);
+    if (CACHED) {
 #pragma unroll
-    for (int r = 0; r < (CACHED ? R : 1); ++r) {
-      for (int rr = (CACHED ? r : 0); rr < (CACHED ? r + 1 : rounds); ++rr) {
-        const int i = w_begin + rr * 32 + lane;
-        const uint32_t u = CACHED ? key[r] : ((i < c_end) ? order_key(__ldg(S + i)) : 0u);
-        const bool is_eq = i < c_end && u == tau;
-        const uint32_t be = __ballot_sync(0xffffffffu, is_eq);
-        const bool keep = i < c_end && (u > tau || (is_eq && eq_run + __popc(be & lt_mask) < need_eq));
-        const uint32_t bk = __ballot_sync(0xffffffffu, keep);
-        if (keep) out[pos + __popc(bk & lt_mask)] = i;
-        pos += __popc(bk);
-        eq_run += __popc(be);
+      for (int r = 0; r < R; ++r) {
+        if (r < n_mine) {
+          const uint32_t u = key[r];
+          const bool is_eq = u == tau;
+          if (u > tau || (is_eq && eq_rank < need_eq)) out[pos++] = t_begin + r;
+          eq_rank += is_eq ? 1 : 0;
+        }
+      }
+    } else {
+      for (int i = t_begin; i < t_end; ++i) {
+        const uint32_t u = order_key(__ldg(S + i));
+        const bool is_eq = u == tau;
+        if (u > tau || (is_eq && eq_rank < need_eq)) out[pos++] = i;
+        eq_rank += is_eq ? 1 : 0;
       }
     }
   }
