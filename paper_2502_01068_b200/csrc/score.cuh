@@ -45,6 +45,7 @@ struct FusedParams {
   float scale_log2;
   const int* cu_seqlens;
   int max_lead;               // phases the HBM pipeline may run ahead of the re-read pipeline
+  int heads_per_phase;        // KV heads of a sequence processed side by side in one phase
   float* a_out;               // [Hkv or Hq][ld_a] un-pooled scores
   long long ld_a;
   float2* partial;            // [phases][CTAs][NPAD]

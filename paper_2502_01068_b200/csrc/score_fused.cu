@@ -42,7 +42,7 @@ struct FusedCfg {
   static constexpr int kTmemCols = 2 * kAcc * NPAD;                         // 256 or 512
   static constexpr int kBarBytes = 512;
   static constexpr int kSmemBytes = 1024 + (kStages1 + kStages2) * kStageBytes + 3 * kQBytes + kBarBytes +
-                                    4 * NPAD * 8 + NPAD * 8 + kGroupWarps * 32 * 8;
+                                    4 * NPAD * 8 + NPAD * 8 + kGroupWarps * 32 * 8 + NPAD * 4;
 };
 
 struct FusedBarriers {
@@ -92,22 +92,33 @@ __device__ __forceinline__ void add_heads(const float (&pr)[16], float (&a_h)[8]
   for (int x = 0; x < 16; ++x) a_h[x % GG] += pr[x];
 }
 
-// what one CTA does in one phase
+// What one CTA does in one phase.  A phase covers `heads_per_phase` KV heads of one sequence; the CTAs
+// are split evenly among those heads (short sequences: fewer, fuller phases), and within a head every
+// CTA owns a run of consecutive tiles.
 struct PhaseWork {
   int b, g, row0, L, t0, n, nact;
+  int stat;                    // index of the (sequence, head) statistics: b * n_kv_heads + g
+  int c;                       // this CTA's index among the CTAs of its head
 };
 
 __device__ __forceinline__ PhaseWork phase_work(const FusedParams& p, int phase, int cta, int ncta) {
   PhaseWork w;
-  w.b = phase / p.n_kv_heads;
-  w.g = phase - w.b * p.n_kv_heads;
+  const int hp = p.heads_per_phase;
+  const int groups = (p.n_kv_heads + hp - 1) / hp;          // phases per sequence
+  w.b = phase / groups;
+  const int g0 = (phase - w.b * groups) * hp;
+  const int ctas_per_head = ncta / hp;
+  const int hi = cta / ctas_per_head;
+  w.c = cta - hi * ctas_per_head;
+  w.g = g0 + hi;
+  w.stat = w.b * p.n_kv_heads + w.g;
   w.row0 = p.cu_seqlens ? p.cu_seqlens[w.b] : 0;
   w.L = p.cu_seqlens ? p.cu_seqlens[w.b + 1] - w.row0 : p.total_len;
-  if (w.L < p.window) { w.t0 = 0; w.n = 0; w.nact = 0; return w; }
+  if (hi >= hp || w.g >= p.n_kv_heads || w.L < p.window) { w.t0 = 0; w.n = 0; w.nact = 0; return w; }
   const int ntiles = (w.L + kTileKeys - 1) / kTileKeys;
-  const int per = (ntiles + ncta - 1) / ncta;
+  const int per = (ntiles + ctas_per_head - 1) / ctas_per_head;
   w.nact = (ntiles + per - 1) / per;
-  w.t0 = cta * per;
+  w.t0 = w.c * per;
   w.n = max(0, min(per, ntiles - w.t0));
   return w;
 }
@@ -134,11 +145,12 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   float2* warp_stats = reinterpret_cast<float2*>(reinterpret_cast<uint8_t*>(bars) + Cfg::kBarBytes);   // [4][NPAD]
   float2* norm = warp_stats + 4 * NPAD;                               // [NPAD] (row max, 1 / row sum)
   float2* merge_buf = norm + NPAD;                                    // [256] partial merges
+  int* row_j = reinterpret_cast<int*>(merge_buf + kGroupWarps * 32);  // [NPAD] window row j = n / G of query row n
   constexpr int CPW = NPAD / 2;                                       // accumulator columns per epilogue warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, ncta = gridDim.x;
-  const int n_phases = p.batch * p.n_kv_heads;
+  const int n_phases = p.batch * ((p.n_kv_heads + p.heads_per_phase - 1) / p.heads_per_phase);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::kStages1; ++s) { mbar_init(&bars->full1[s], 1); mbar_init(&bars->empty1[s], 1); }
@@ -163,6 +175,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     tmem_alloc(&bars->tmem_base, Cfg::kTmemCols);
     tmem_relinquish();
   }
+  if (threadIdx.x >= 64 && threadIdx.x < 64 + NPAD) row_j[threadIdx.x - 64] = (threadIdx.x - 64) / p.group;   // divide once
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -304,7 +317,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             if (key < w.L) {
 #pragma unroll
               for (int x = 0; x < 16; ++x)
-                if (x < n_valid && key <= win_start + (col0 + c * 16 + x) / G) visible |= 1u << x;
+                if (x < n_valid && key <= win_start + row_j[col0 + c * 16 + x]) visible |= 1u << x;
             }
             stats_update_masked<16>(acc, m + c * 16, l + c * 16, p.scale_log2, n_valid, visible);
           }
@@ -322,12 +335,12 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         float mm = -INFINITY, ll = 0.0f;
 #pragma unroll
         for (int q = 0; q < 4; ++q) merge_stats(mm, ll, warp_stats[q * NPAD + at].x, warp_stats[q * NPAD + at].y);
-        p.partial[(static_cast<size_t>(phase) * ncta + cta) * NPAD + at] = make_float2(mm, ll);
+        p.partial[(static_cast<size_t>(w.stat) * ncta + w.c) * NPAD + at] = make_float2(mm, ll);
       }
       group_sync<1>();                                   // also: warp_stats may be rewritten next phase
       ++u;
       if (at == 0) {
-        red_release_add(p.counters + phase, 1);          // release: cumulative over the barrier
+        red_release_add(p.counters + w.stat, 1);         // release: cumulative over the barrier
         bars->p1_done = u;                               // pipeline 2 may re-read this phase's tiles
       }
     }
@@ -350,7 +363,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       if (w.n == 0) continue;
       // every CTA that owns tiles of this phase has published its statistics?
       if (bt == 0) {
-        const int* ctr = p.counters + phase;
+        const int* ctr = p.counters + w.stat;
         if (ld_acquire(ctr) < w.nact) {
           const long long t0 = clock64();
           unsigned spins = 0;
@@ -366,7 +379,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       group_sync<2>();
       if (*abort_flag) break;
       // the softmax normaliser of the phase, merged in a fixed order (the same in every CTA)
-      merge_buf[bt] = merge_partials(p.partial + static_cast<size_t>(phase) * ncta * NPAD, NPAD, bt % NPAD, bt / NPAD,
+      merge_buf[bt] = merge_partials(p.partial + static_cast<size_t>(w.stat) * ncta * NPAD, NPAD, bt % NPAD, bt / NPAD,
                                      kParts, w.nact);
       group_sync<2>();
       if (bt < NPAD) {
@@ -409,7 +422,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           if (!tile_unmasked) {                          // causal: key i <= t_j, j = n / G
 #pragma unroll
             for (int x = 0; x < 16; ++x)
-              if (x < n_valid && key > win_start + (c * 16 + x) / G) pr[x] = 0.0f;
+              if (x < n_valid && key > win_start + row_j[c * 16 + x]) pr[x] = 0.0f;
           }
           if (!p.per_head) {
 #pragma unroll
