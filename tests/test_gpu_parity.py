@@ -138,3 +138,16 @@ def test_wide_logit_range_exercises_reference_rescaling(scale):
         assert np.all(np.abs(got - ref_kv) <= SCORE_RTOL * np.abs(ref_kv) + 1e-12)
         np.testing.assert_allclose(got.sum(axis=1), ref_kv.sum(axis=1), rtol=1e-5)
         assert np.all(np.abs(s_tsp.cpu().numpy() - ref_tsp) <= SCORE_RTOL * np.abs(ref_tsp) + 1e-12)
+
+
+@pytest.mark.parametrize("heads,lead", [("1", "2"), ("2", "1000"), ("3", "2"), ("8", "3")])
+def test_phase_shapes_of_the_scoring_kernel(monkeypatch, heads, lead):
+    """The persistent scoring kernel cuts its work into phases of `heads` KV heads and lets pass 1 run
+    `lead` phases ahead; the result must not depend on either (tuning knobs forced through the environment)."""
+    monkeypatch.setenv("FASTKV_FUSED_HEADS", heads)
+    monkeypatch.setenv("FASTKV_FUSED_LEAD", lead)
+    wl = small("phases", 900, [20000, 3000], [500, 100], [2000, 300], Hq=32, Hkv=8)
+    x = W.make_layer(wl, with_hidden=False)
+    g = gpu_layer(wl, x)
+    o = oracle_layer(wl, x, do_compact=False)
+    check_layer(wl, x, g, o, what="heads=%s lead=%s" % (heads, lead))
