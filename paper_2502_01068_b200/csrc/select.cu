@@ -45,8 +45,11 @@ struct alignas(16) SelShared {
 // and the ordered compaction at the end needs no warp votes, only one scan of per-thread counts.
 // ITEMS > 0: per = ITEMS and the candidates (converted once) stay in registers for all passes.
 // ITEMS == 0: any chunk size; every pass re-reads the scores (they are L2 resident).
-template <int CLUSTER, int ITEMS>
-__global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const SelectParams p) {
+template <int CLUSTER, int ITEMS, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1) select_topk_kernel(const SelectParams p) {
+  constexpr int kWarps = THREADS / 32;
+  constexpr int kPerBin = THREADS / kBins;         // threads that share one bin in the histogram reduction
+  static_assert(THREADS % kBins == 0 && kPerBin >= 1 && kPerBin <= 4, "256, 512 or 1024 threads");
   cg::cluster_group cluster = cg::this_cluster();
   __shared__ SelShared sh;
   constexpr bool CACHED = ITEMS > 0;
@@ -79,7 +82,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
   // contiguous chunk per CTA, `per` consecutive candidates per thread
   const int chunk = ((n_cand + CLUSTER - 1) / CLUSTER + 3) & ~3;   // multiple of 4: keeps 16-byte alignment
   const int c_begin = min(n_cand, rank * chunk), c_end = min(n_cand, c_begin + chunk);
-  const int per = CACHED ? ITEMS : (chunk + kSelThreads - 1) / kSelThreads;
+  const int per = CACHED ? ITEMS : (chunk + THREADS - 1) / THREADS;
   const int t_begin = min(c_end, c_begin + tid * per), t_end = min(c_end, t_begin + per);
   const int n_mine = t_end - t_begin;
 
@@ -103,7 +106,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
   uint32_t prefix = 0;
   int k_rem = k_sel;
   if (k_sel > 0) {
-    for (int i = tid; i < kBins * 32; i += kSelThreads) sh.hist[i] = 0;
+    for (int i = tid; i < kBins * 32; i += THREADS) sh.hist[i] = 0;
     __syncthreads();
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
@@ -122,17 +125,17 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
       }
       __syncthreads();
       {
-        // 4 threads per bin, each sums (and clears for the next pass) 8 lane counters
-        const int bin = tid >> 2, part = tid & 3;
+        // kPerBin threads per bin, each sums (and clears for the next pass) its share of the 32 lane counters
+        const int bin = tid / kPerBin, part = tid % kPerBin;
         int sum = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          int* c = &sh.hist[bin * 32 + ((part * 8 + i + bin) & 31)];
+        for (int i = 0; i < 32 / kPerBin; ++i) {
+          int* c = &sh.hist[bin * 32 + ((part * (32 / kPerBin) + i + bin) & 31)];
           sum += *c;
           *c = 0;
         }
-        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        if (kPerBin >= 2) sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        if (kPerBin >= 4) sum += __shfl_xor_sync(0xffffffffu, sum, 2);
         if (part == 0) sh.block_hist[pass & 1][bin] = sum;
       }
       cluster.sync();
@@ -213,7 +216,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
   if (lane == 31) { sh.warp_tot[0][warp] = gt_incl; sh.warp_tot[1][warp] = eq_incl; }
   __syncthreads();
   if (warp == 0) {
-    int a = sh.warp_tot[0][lane], e = sh.warp_tot[1][lane];
+    int a = lane < kWarps ? sh.warp_tot[0][lane] : 0, e = lane < kWarps ? sh.warp_tot[1][lane] : 0;
     const int a0 = a, e0 = e;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -271,12 +274,12 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const Selec
 
 namespace {
 
-template <int CLUSTER, int ITEMS>
+template <int CLUSTER, int ITEMS, int THREADS>
 cudaError_t launch_select_t(const SelectParams& p, int batch, cudaStream_t stream) {
   if (CLUSTER > 8) {
     static bool configured = false;
     if (!configured) {
-      cudaError_t e = cudaFuncSetAttribute(select_topk_kernel<CLUSTER, ITEMS>,
+      cudaError_t e = cudaFuncSetAttribute(select_topk_kernel<CLUSTER, ITEMS, THREADS>,
                                            cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
       if (e != cudaSuccess) return e;
       configured = true;
@@ -284,7 +287,7 @@ cudaError_t launch_select_t(const SelectParams& p, int batch, cudaStream_t strea
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(CLUSTER, p.set[0].n_rows + p.set[1].n_rows, batch);
-  cfg.blockDim = dim3(kSelThreads);
+  cfg.blockDim = dim3(THREADS);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
@@ -295,20 +298,31 @@ cudaError_t launch_select_t(const SelectParams& p, int batch, cudaStream_t strea
   fill_pdl_attribute(&attr[1]);
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, select_topk_kernel<CLUSTER, ITEMS>, p);
+  return cudaLaunchKernelEx(&cfg, select_topk_kernel<CLUSTER, ITEMS, THREADS>, p);
 }
 
 }  // namespace
 
+template <int CLUSTER, int THREADS>
+static cudaError_t launch_select_c(const SelectParams& p, int batch, int max_len, cudaStream_t stream) {
+  const long long per_cta = (static_cast<long long>(max_len) + CLUSTER - 1) / CLUSTER;
+  if (per_cta <= 4 * THREADS) return launch_select_t<CLUSTER, 4, THREADS>(p, batch, stream);
+  if (per_cta <= 8 * THREADS) return launch_select_t<CLUSTER, 8, THREADS>(p, batch, stream);
+  if (per_cta <= 16 * THREADS) return launch_select_t<CLUSTER, 16, THREADS>(p, batch, stream);
+  if (per_cta <= 32 * THREADS) return launch_select_t<CLUSTER, 32, THREADS>(p, batch, stream);
+  return launch_select_t<CLUSTER, 0, THREADS>(p, batch, stream);
+}
+
 cudaError_t launch_select(const SelectParams& p, int batch, int max_len, cudaStream_t stream) {
-  // 8-CTA clusters: every problem of a layer (KV heads plus the TSP row) is resident at once on a
-  // 148-SM part.  The per-thread register cache is picked from the longest sequence.
-  const long long per_cta = (static_cast<long long>(max_len) + 7) / 8;
-  if (per_cta <= 4 * kSelThreads) return launch_select_t<8, 4>(p, batch, stream);
-  if (per_cta <= 8 * kSelThreads) return launch_select_t<8, 8>(p, batch, stream);
-  if (per_cta <= 16 * kSelThreads) return launch_select_t<8, 16>(p, batch, stream);
-  if (per_cta <= 32 * kSelThreads) return launch_select_t<8, 32>(p, batch, stream);
-  return launch_select_t<8, 0>(p, batch, stream);
+  // Long sequences: 8-CTA clusters of 1024 threads, with which every problem of a layer (KV heads plus the
+  // TSP row) is resident at once on a 148-SM part.  Short sequences are bound by the fixed cost of the CTA
+  // and cluster barriers, so they use 256-thread CTAs (16 candidates per thread) in clusters as small as
+  // the length allows.  The per-thread register cache is picked from the longest sequence.
+  if (max_len <= 16 * 256) return launch_select_c<1, 256>(p, batch, max_len, stream);
+  if (max_len <= 2 * 16 * 256) return launch_select_c<2, 256>(p, batch, max_len, stream);
+  if (max_len <= 4 * 16 * 256) return launch_select_c<4, 256>(p, batch, max_len, stream);
+  if (max_len <= 8 * 16 * 256) return launch_select_c<8, 256>(p, batch, max_len, stream);
+  return launch_select_c<8, 1024>(p, batch, max_len, stream);
 }
 
 }  // namespace fastkv
