@@ -280,15 +280,15 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
     // A phase is sized to about one head of a 128K-token sequence (33.5 MB of K): shorter sequences put several
     // heads side by side in a phase, so that there are fewer grid-wide dependencies per byte.  Pass 1 may lead pass 2
     // by as many phases as keep about 110 MB of K between the two reads: that is what stays in the 126 MB L2.
-    const double head_bytes = static_cast<double>(s.max_len) * s.head_dim * 2.0;
     const char* hpp = std::getenv("FASTKV_FUSED_HEADS");     // tuning knobs
     const char* lead = std::getenv("FASTKV_FUSED_LEAD");
-    int hp = hpp ? std::atoi(hpp) : static_cast<int>(35e6 / head_bytes);
-    if (hp > s.n_kv_heads) hp = s.n_kv_heads;
-    if (hp > ctas) hp = ctas;
-    if (hp < 1) hp = 1;
-    fp.heads_per_phase = hp;
-    fp.max_lead = lead ? std::atoi(lead) : static_cast<int>(110e6 / (head_bytes * hp));
+    fp.heads_per_phase = hpp ? std::atoi(hpp) : 0;
+    fp.phase_bytes = 35000000;
+    fp.head_bytes = static_cast<long long>(s.head_dim) * 2;
+    double longest_phase = static_cast<double>(s.max_len) * s.head_dim * 2.0;     // bytes of the largest phase
+    const double hp_longest = fp.heads_per_phase > 0 ? fp.heads_per_phase : fp.phase_bytes / longest_phase;
+    if (hp_longest >= 1.0) longest_phase *= static_cast<int>(hp_longest < s.n_kv_heads ? hp_longest : s.n_kv_heads);
+    fp.max_lead = lead ? std::atoi(lead) : static_cast<int>(110e6 / longest_phase);
     if (fp.max_lead > (1 << 20)) fp.max_lead = 1 << 20;
     if (fp.max_lead < 2) fp.max_lead = 2;
     fp.partial = reinterpret_cast<float2*>(ws + lay.f_off_partial);

@@ -45,7 +45,10 @@ struct FusedParams {
   float scale_log2;
   const int* cu_seqlens;
   int max_lead;               // phases the HBM pipeline may run ahead of the re-read pipeline
-  int heads_per_phase;        // KV heads of a sequence processed side by side in one phase
+  int heads_per_phase;        // > 0: KV heads of a sequence processed side by side in one phase (forced);
+                              // 0: chosen per sequence so that a phase holds about phase_bytes of K
+  long long phase_bytes;      // target size of a phase
+  long long head_bytes;       // bytes of one key row of one head (head_dim * 2)
   float* a_out;               // [Hkv or Hq][ld_a] un-pooled scores
   long long ld_a;
   float2* partial;            // [phases][CTAs][NPAD]

@@ -92,35 +92,46 @@ __device__ __forceinline__ void add_heads(const float (&pr)[16], float (&a_h)[8]
   for (int x = 0; x < 16; ++x) a_h[x % GG] += pr[x];
 }
 
-// What one CTA does in one phase.  A phase covers `heads_per_phase` KV heads of one sequence; the CTAs
-// are split evenly among those heads (short sequences: fewer, fuller phases), and within a head every
-// CTA owns a run of consecutive tiles.
+// What one CTA does in one phase.  A phase covers a few KV heads of one sequence -- as many as keep it
+// near `phase_bytes` of K, so short sequences get fewer, fuller phases and fewer grid-wide
+// dependencies; the CTAs are split evenly among those heads, and within a head every CTA owns a run
+// of consecutive tiles.  Every role of every CTA walks the same sequence of phases.
 struct PhaseWork {
   int b, g, row0, L, t0, n, nact;
   int stat;                    // index of the (sequence, head) statistics: b * n_kv_heads + g
   int c;                       // this CTA's index among the CTAs of its head
 };
 
-__device__ __forceinline__ PhaseWork phase_work(const FusedParams& p, int phase, int cta, int ncta) {
-  PhaseWork w;
-  const int hp = p.heads_per_phase;
-  const int groups = (p.n_kv_heads + hp - 1) / hp;          // phases per sequence
-  w.b = phase / groups;
-  const int g0 = (phase - w.b * groups) * hp;
-  const int ctas_per_head = ncta / hp;
+struct PhaseIter {
+  int b, g0;                   // next phase: sequence b, heads g0 .. g0 + hp - 1
+};
+
+__device__ __forceinline__ bool next_phase(const FusedParams& p, PhaseIter& it, int cta, int ncta, PhaseWork& w) {
+  if (it.b >= p.batch) return false;
+  w.b = it.b;
+  w.row0 = p.cu_seqlens ? p.cu_seqlens[w.b] : 0;
+  w.L = p.cu_seqlens ? p.cu_seqlens[w.b + 1] - w.row0 : p.total_len;
+  // heads per phase of this sequence: the same arithmetic in every thread that walks the phases
+  long long hp = p.phase_bytes / (static_cast<long long>(w.L > 0 ? w.L : 1) * p.head_bytes);
+  if (p.heads_per_phase > 0) hp = p.heads_per_phase;        // forced
+  if (hp > p.n_kv_heads) hp = p.n_kv_heads;
+  if (hp > ncta) hp = ncta;
+  if (hp < 1) hp = 1;
+  const int g0 = it.g0;
+  it.g0 += static_cast<int>(hp);
+  if (it.g0 >= p.n_kv_heads) { it.g0 = 0; ++it.b; }
+  const int ctas_per_head = ncta / static_cast<int>(hp);
   const int hi = cta / ctas_per_head;
   w.c = cta - hi * ctas_per_head;
   w.g = g0 + hi;
   w.stat = w.b * p.n_kv_heads + w.g;
-  w.row0 = p.cu_seqlens ? p.cu_seqlens[w.b] : 0;
-  w.L = p.cu_seqlens ? p.cu_seqlens[w.b + 1] - w.row0 : p.total_len;
-  if (hi >= hp || w.g >= p.n_kv_heads || w.L < p.window) { w.t0 = 0; w.n = 0; w.nact = 0; return w; }
+  if (hi >= hp || w.g >= p.n_kv_heads || w.L < p.window) { w.t0 = 0; w.n = 0; w.nact = 0; return true; }
   const int ntiles = (w.L + kTileKeys - 1) / kTileKeys;
   const int per = (ntiles + ctas_per_head - 1) / ctas_per_head;
   w.nact = (ntiles + per - 1) / per;
   w.t0 = w.c * per;
   w.n = max(0, min(per, ntiles - w.t0));
-  return w;
+  return true;
 }
 
 }  // namespace
@@ -150,7 +161,6 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, ncta = gridDim.x;
-  const int n_phases = p.batch * ((p.n_kv_heads + p.heads_per_phase - 1) / p.heads_per_phase);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::kStages1; ++s) { mbar_init(&bars->full1[s], 1); mbar_init(&bars->empty1[s], 1); }
@@ -199,8 +209,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       const int nq = second ? 1 : 2;                     // Q buffers of the pipeline
       int it = 0, u = 0;
       bool ok = true;
-      for (int phase = 0; ok && phase < n_phases; ++phase) {
-        const PhaseWork w = phase_work(p, phase, cta, ncta);
+      PhaseIter pit = {0, 0};
+      PhaseWork w;
+      while (ok && next_phase(p, pit, cta, ncta, w)) {
         if (w.n == 0) continue;
         // pipeline 2 re-reads what pipeline 1 of this CTA has finished with; pipeline 1 stays close
         // enough ahead for those tiles to be still in L2
@@ -244,8 +255,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       const uint32_t acc_base = tmem_base + (second ? kAcc * NPAD : 0);
       int it = 0, u = 0;
       bool ok = true;
-      for (int phase = 0; ok && phase < n_phases; ++phase) {
-        const PhaseWork w = phase_work(p, phase, cta, ncta);
+      PhaseIter pit = {0, 0};
+      PhaseWork w;
+      while (ok && next_phase(p, pit, cta, ncta, w)) {
         if (w.n == 0) continue;
         const int h = u % nq;
         ok = mbar_wait_bounded(&q_full[h], (u / nq) & 1, abort_flag, p.hdr, SITE_FUSED_Q_FULL);
@@ -284,8 +296,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + col0;
     int it = 0, u = 0;
     bool ok = true;
-    for (int phase = 0; ok && phase < n_phases; ++phase) {
-      const PhaseWork w = phase_work(p, phase, cta, ncta);
+    PhaseIter pit = {0, 0};
+    PhaseWork w;
+    while (ok && next_phase(p, pit, cta, ncta, w)) {
       if (w.n == 0) continue;
       float m[CPW], l[CPW];
 #pragma unroll
@@ -358,8 +371,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     constexpr int kParts = kGroupWarps * 32 / NPAD;
     int it = 0, u = 0;
     bool ok = true;
-    for (int phase = 0; ok && phase < n_phases; ++phase) {
-      const PhaseWork w = phase_work(p, phase, cta, ncta);
+    PhaseIter pit = {0, 0};
+    PhaseWork w;
+    while (ok && next_phase(p, pit, cta, ncta, w)) {
       if (w.n == 0) continue;
       // every CTA that owns tiles of this phase has published its statistics?
       if (bt == 0) {
