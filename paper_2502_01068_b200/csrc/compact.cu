@@ -12,7 +12,7 @@ namespace {
 
 constexpr int kChunkBytes = 8192;
 constexpr int kStages = 4;                 // chunks in flight per warp
-constexpr int kCompactWarps = 6;
+constexpr int kCompactWarps = 7;                 // 7 x 4 x 8 KB = 224 KB of shared memory per CTA
 constexpr int kCompactThreads = kCompactWarps * 32;
 constexpr int kCompactSmem = kCompactWarps * kStages * kChunkBytes + 1024;
 
