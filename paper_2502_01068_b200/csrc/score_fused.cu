@@ -299,7 +299,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     PhaseIter pit = {0, 0};
     PhaseWork w;
     while (ok && next_phase(p, pit, cta, ncta, w)) {
-      if (w.n == 0) continue;
+      if (w.n == 0) {
+        // a sequence shorter than the observation window has no defined scores: say so once
+        if (w.L < p.window && cta == 0 && at == 0) raise_status(p.hdr, FASTKV_ERR_INVALID_ARG, SITE_SCORE_SHORT_SEQUENCE);
+        continue;
+      }
       float m[CPW], l[CPW];
 #pragma unroll
       for (int n = 0; n < CPW; ++n) { m[n] = -INFINITY; l[n] = 0.0f; }

@@ -151,3 +151,26 @@ def test_phase_shapes_of_the_scoring_kernel(monkeypatch, heads, lead):
     g = gpu_layer(wl, x)
     o = oracle_layer(wl, x, do_compact=False)
     check_layer(wl, x, g, o, what="heads=%s lead=%s" % (heads, lead))
+
+
+def test_sequence_shorter_than_the_window_is_reported_not_scored():
+    """In a batch, a sequence with fewer tokens than the observation window has no defined scores: the
+    scoring kernel skips it and raises the status word; the other sequences are unaffected."""
+    lens = [300, 5, 700]
+    wl = small("short", 950, lens, [40, 8, 60], [50, 8, 90])
+    x = W.make_layer(wl, with_hidden=False)
+    from tests.parity import dev
+    cu = dev(x.cu_seqlens.astype(np.int32))
+    shape = B.make_shape(total_len=sum(lens), n_q_heads=8, n_kv_heads=2, head_dim=128, batch=3, max_len=700,
+                         cu_seqlens=cu)
+    ws = torch.empty(B.fastkv_workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+    s_kv = torch.zeros((2, sum(lens)), dtype=torch.float32, device="cuda")
+    B.fastkv_score(shape, dev(x.q_win), dev(x.k), s_kv, None, ws)
+    status, site = B.fastkv_device_status(ws)
+    assert status == B.ERR_INVALID_ARG
+    import oracle
+    got = s_kv.cpu().numpy()
+    for b in (0, 2):
+        lo, hi = int(x.cu_seqlens[b]), int(x.cu_seqlens[b + 1])
+        ref, _, _ = oracle.scores(x.q_win[b * 8:(b + 1) * 8], hi - lo - 8, x.k[lo:hi], 8, 7)
+        assert np.all(np.abs(got[:, lo:hi] - ref) <= 2e-3 * np.abs(ref) + 1e-12)
