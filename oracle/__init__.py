@@ -43,6 +43,7 @@ def _load():
                                       vp, vp, vp]
         lib.oracle_select.argtypes = [vp, i64, i64, i32, i32, vp, vp]
         lib.oracle_gather_rows.argtypes = [vp, i64, i64, vp, i64, vp]
+        lib.oracle_decode_attention.argtypes = [vp, vp, vp, i64, i32, i32, i32, f64, vp, vp]
         lib.oracle_num_threads.restype = i32
         _lib = lib
     return _lib
@@ -138,3 +139,18 @@ def gather_rows(src: np.ndarray, idx: np.ndarray) -> np.ndarray:
     _load().oracle_gather_rows(_ptr(src), src.strides[0], row_bytes, _ptr(idx), idx.shape[0],
                                _ptr(dst))
     return dst
+
+
+def decode_attention(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray, scale: Optional[float] = None):
+    """One query token over a compressed cache: q [H, d], k_cache / v_cache [Hkv, k, d] (bf16 bits).
+    Returns (out [H, d] fp64, lse [H] fp64)."""
+    q, k_cache, v_cache = _u16(q), _u16(k_cache), _u16(v_cache)
+    H, d = q.shape
+    Hkv, k, _ = k_cache.shape
+    out = np.empty((H, d), dtype=np.float64)
+    lse = np.empty((H,), dtype=np.float64)
+    rc = _load().oracle_decode_attention(_ptr(q), _ptr(k_cache), _ptr(v_cache), k, H, Hkv, d,
+                                         (d ** -0.5) if scale is None else scale, _ptr(out), _ptr(lse))
+    if rc:
+        raise ValueError("oracle_decode_attention rejected its arguments")
+    return out, lse

@@ -28,7 +28,8 @@
  * Parity pins (tests/test_oracle_*.py): full LxL causal attention through a
  * library softmax, the uniform-attention and single-planted-key closed forms,
  * row-sum / shift / permutation invariants, pooling identities, selection
- * against a brute-force ranking, gather against numpy indexing.  Nothing
+ * against a brute-force ranking, gather against numpy indexing, decode attention against a
+ * library softmax-attention and closed forms.  Nothing
  * numeric from the paper's own implementation exists to compare against, so
  * parity with that implementation is unpinned; parity with the definitions
  * above is pinned.
@@ -260,6 +261,43 @@ int oracle_gather_rows(const uint8_t* src, int64_t src_stride_bytes, int64_t row
                        const int64_t* idx, int64_t n, uint8_t* dst) {
     for (int64_t j = 0; j < n; ++j)
         memcpy(dst + j * row_bytes, src + idx[j] * src_stride_bytes, (size_t)row_bytes);
+    return 0;
+}
+
+/*
+ * Decoding over the compressed cache (the stage the retained KV of Alg. 1 exists for; Sec. 3, Sec. 5.3):
+ * one new query token attends to the k retained entries of its KV group.
+ *   out[h, :] = sum_j softmax_j(scale * <q[h], K[h/G, j]>) * V[h/G, j, :],   j = 0..k-1
+ * q is [H, d], k_cache and v_cache are [Hkv, k, d] (bf16 bits, dense), out is [H, d] fp64, lse (optional)
+ * is the natural-log sum of exponentials of each head's logits.
+ */
+int oracle_decode_attention(const uint16_t* q, const uint16_t* k_cache, const uint16_t* v_cache, int64_t k,
+                            int H, int Hkv, int d, double scale, double* out, double* lse) {
+    if (k < 1 || H % Hkv != 0) return 1;
+    const int G = H / Hkv;
+    double* s = (double*)malloc((size_t)k * sizeof(double));
+    if (!s) return 1;
+    for (int h = 0; h < H; ++h) {
+        const int g = h / G;
+        double smax = -INFINITY;
+        for (int64_t j = 0; j < k; ++j) {
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c)
+                acc += bf16_to_f64(q[(int64_t)h * d + c]) * bf16_to_f64(k_cache[((int64_t)g * k + j) * d + c]);
+            s[j] = scale * acc;
+            if (s[j] > smax) smax = s[j];
+        }
+        double denom = 0.0;
+        for (int64_t j = 0; j < k; ++j) denom += exp(s[j] - smax);
+        for (int c = 0; c < d; ++c) {
+            double acc = 0.0;
+            for (int64_t j = 0; j < k; ++j)
+                acc += exp(s[j] - smax) / denom * bf16_to_f64(v_cache[((int64_t)g * k + j) * d + c]);
+            out[(int64_t)h * d + c] = acc;
+        }
+        if (lse) lse[h] = smax + log(denom);
+    }
+    free(s);
     return 0;
 }
 

@@ -309,3 +309,35 @@ def test_layer_step_ragged_batch_equals_per_sequence_runs():
         np.testing.assert_array_equal(r["pos_out"][a:e], one["pos_out"])
         a, e = r["cu_k_kv"][b], r["cu_k_kv"][b + 1]
         np.testing.assert_array_equal(r["k_out"][:, a:e], one["k_out"])
+
+
+def test_decode_attention_matches_library_attention_and_closed_forms():
+    """The decode step over the compressed cache is plain softmax attention of one query token: pinned
+    against torch's scaled_dot_product_attention in fp64 and against two closed forms."""
+    rng = np.random.default_rng(21)
+    H, Hkv, d, k = 8, 2, 16, 37
+    q = bf16(rng.standard_normal((H, d)))
+    kc = bf16(rng.standard_normal((Hkv, k, d)))
+    vc = bf16(rng.standard_normal((Hkv, k, d)))
+    out, lse = oracle.decode_attention(q, kc, vc)
+    G = H // Hkv
+    tq = torch.from_numpy(f64(q))[None, :, None, :]                               # [1, H, 1, d]
+    tk = torch.from_numpy(f64(kc)).repeat_interleave(G, dim=0)[None]              # head h reads group h // G
+    tv = torch.from_numpy(f64(vc)).repeat_interleave(G, dim=0)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv)[0, :, 0, :].numpy()
+    np.testing.assert_allclose(out, ref, rtol=0, atol=1e-13)
+    logits = torch.einsum("hd,hkd->hk", tq[0, :, 0, :], tk[0]) / math.sqrt(d)
+    np.testing.assert_allclose(lse, torch.logsumexp(logits, dim=-1).numpy(), rtol=0, atol=1e-13)
+    # all keys equal: the output is the mean of the values
+    kc_same = np.broadcast_to(kc[:, :1, :], kc.shape).copy()
+    out_u, lse_u = oracle.decode_attention(q, kc_same, vc)
+    np.testing.assert_allclose(out_u, np.repeat(f64(vc).mean(axis=1), G, axis=0), rtol=0, atol=1e-13)
+    # one key aligned with the query and far above the rest: the output is that key's value row
+    kc_hot = np.zeros_like(kc); kc_hot[:, 5, :] = bf16(40.0 * f64(q)[::G])
+    out_h, _ = oracle.decode_attention(q[::G].repeat(G, axis=0), kc_hot, vc)
+    np.testing.assert_allclose(out_h, np.repeat(f64(vc)[:, 5, :], G, axis=0), rtol=0, atol=1e-9)
+    # permuting cache entries (K and V together) changes nothing
+    perm = rng.permutation(k)
+    out_p, lse_p = oracle.decode_attention(q, kc[:, perm], vc[:, perm])
+    np.testing.assert_allclose(out_p, out, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(lse_p, lse, rtol=0, atol=1e-13)
