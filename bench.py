@@ -227,6 +227,8 @@ def main() -> None:
     ap.add_argument("--impl", default="fastkv", choices=["fastkv", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--with-decode", action="store_true",
+                    help="also time the decode-time attention over the compact cache the step produced")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -370,6 +372,28 @@ def main() -> None:
         if np.array_equal(o_idx_tsp.numpy(), idx_tsp.cpu().numpy()) is False:
             raise SystemExit("host-buffer path and device path disagree on idx_tsp")
 
+    # ---- optional: decode-time attention of one new token over the compacted cache of this layer ------------------
+    decode = None
+    if args.with_decode and len(set(wl.k_kv)) == 1:
+        qd = torch.randn((Bn, wl.n_q_heads, wl.head_dim), device="cuda").to(torch.bfloat16).view(torch.int16)
+        dws = torch.empty(B.fastkv_decode_attn_workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+        dout = torch.empty((Bn, wl.n_q_heads, wl.head_dim), dtype=torch.float32, device="cuda")
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # the cache alone would fit in L2
+        times = []
+        for i in range(13):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            B.fastkv_decode_attn(shape, qd, k_out, v_out, b_kv, dout, None, dws, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                times.append(e0.elapsed_time(e1))
+        dms = statistics.median(times)
+        dbytes = 2 * wl.n_kv_heads * b_kv.total * wl.head_dim * 2
+        decode = {"ms": dms, "algorithmic_bytes": dbytes, "achieved_gbs": dbytes / (dms * 1e-3) / 1e9,
+                  "frac_of_measured": dbytes / (dms * 1e-3) / 1e9 / measured_peaks()["hbm_gbs"],
+                  "l2": "flushed between iterations (256 MB write)", "kept_per_head": int(wl.k_kv[0])}
     if rank != 0:
         return
     ab = algorithmic_bytes(wl)
@@ -401,6 +425,8 @@ def main() -> None:
                      "step_with_events_between_calls": instrumented_ms},
         "calls_gbs": {"fastkv_score": ab["score"] / (call_ms[0] * 1e-3) / 1e9},
     }
+    if decode is not None:
+        line["decode_attn"] = decode
     if not args.no_cpu_baseline:
         line["cpu_baseline"] = oracle_baseline(wl, x)
     print(json.dumps(line))

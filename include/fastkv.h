@@ -155,6 +155,20 @@ int fastkv_compact(const fastkv_shape* shape, const int32_t* idx_kv, const fastk
                    void* stream);
 
 /*
+ * Decoding over the compressed cache (what the retained KV of Alg. 1 is kept for; Sec. 3, Sec. 5.3): one new
+ * query token per sequence attends to the kept entries of its KV group,
+ *   out[b, h, :] = sum_j softmax_j(scale * <q[b, h], K[h / G, j]>) * V[h / G, j, :],  j over sequence b's kept entries.
+ * q: bf16 [B, n_q_heads, head_dim]; k_cache, v_cache: bf16 [n_kv_heads, kv.total, head_dim], the k_out / v_out
+ * layout of fastkv_compact; out: fp32 [B, n_q_heads, head_dim]; lse (optional): fp32 [B, n_q_heads], natural-log
+ * sum of exponentials of each head's logits.  workspace: >= fastkv_decode_attn_workspace_bytes, 256-byte aligned
+ * (the status word is not cleared by this call).  head_dim 64 or 128, at most 8 query heads per KV head.
+ */
+int fastkv_decode_attn_workspace_bytes(const fastkv_shape* shape, size_t* bytes);
+int fastkv_decode_attn(const fastkv_shape* shape, const void* q, const void* k_cache, const void* v_cache,
+                       const fastkv_budget* kv, float* out, float* lse, void* workspace, size_t workspace_bytes,
+                       void* stream);
+
+/*
  * Synchronises `stream`, then copies the device status word of `workspace` to the HOST
  * integers *status (a fastkv_status) and *site (which wait or check raised it; 0 if none).
  */

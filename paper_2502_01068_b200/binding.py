@@ -21,7 +21,7 @@ GROUP_THEN_POOL, POOL_THEN_GROUP = 0, 1
 Q_FULL, Q_WINDOW = 0, 1
 
 EXPORTS = ["fastkv_workspace_bytes", "fastkv_score", "fastkv_select_kv", "fastkv_select_tsp", "fastkv_select",
-           "fastkv_compact", "fastkv_device_status", "fastkv_layer_host_arena_bytes",
+           "fastkv_compact", "fastkv_decode_attn_workspace_bytes", "fastkv_decode_attn", "fastkv_device_status", "fastkv_layer_host_arena_bytes",
            "fastkv_layer_host", "fastkv_score_static", "fastkv_status_string", "fastkv_last_error",
            "fastkv_kernel_launches"]
 
@@ -81,7 +81,9 @@ def _load():
         lib.fastkv_last_error.restype = ctypes.c_char_p
         lib.fastkv_kernel_launches.restype = ctypes.c_int64
         lib.fastkv_score_static.argtypes = [ps, vp, vp, vp, vp, vp]
-        for fn in EXPORTS[:10]:
+        lib.fastkv_decode_attn_workspace_bytes.argtypes = [ps, ctypes.POINTER(sz)]
+        lib.fastkv_decode_attn.argtypes = [ps, vp, vp, vp, pb, vp, vp, vp, sz, vp]
+        for fn in EXPORTS[:12]:
             getattr(lib, fn).restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -180,6 +182,19 @@ def fastkv_compact(shape: Shape, idx_kv, kv: Optional[Budget], idx_tsp, tsp: Opt
                                   _p(pos_ids), _p(k_out), _p(v_out), _p(hidden_out), _p(pos_out),
                                   _p(workspace), workspace.numel() * workspace.element_size(),
                                   _stream(stream)), "fastkv_compact")
+
+
+def fastkv_decode_attn_workspace_bytes(shape: Shape) -> int:
+    n = ctypes.c_size_t(0)
+    _check(_load().fastkv_decode_attn_workspace_bytes(ctypes.byref(shape), ctypes.byref(n)),
+           "fastkv_decode_attn_workspace_bytes")
+    return int(n.value)
+
+
+def fastkv_decode_attn(shape: Shape, q, k_cache, v_cache, kv: Budget, out, lse, workspace, stream=None) -> None:
+    _check(_load().fastkv_decode_attn(ctypes.byref(shape), _p(q), _p(k_cache), _p(v_cache), ctypes.byref(kv), _p(out),
+                                      _p(lse), _p(workspace), workspace.numel() * workspace.element_size(),
+                                      _stream(stream)), "fastkv_decode_attn")
 
 
 def fastkv_device_status(workspace, stream=None):

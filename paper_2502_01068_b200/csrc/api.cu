@@ -8,6 +8,7 @@
 #include <cstring>
 
 #include "compact.cuh"
+#include "decode_attn.cuh"
 #include "score.cuh"
 #include "select.cuh"
 
@@ -455,6 +456,50 @@ int fastkv_compact(const fastkv_shape* shape, const int32_t* idx_kv, const fastk
   cudaError_t e = launch_compact(cp, static_cast<cudaStream_t>(stream_));
   if (e != cudaSuccess) return cuda_fail(e, "compact_rows_kernel launch");
   ++g_launches;
+  return FASTKV_OK;
+}
+
+int fastkv_decode_attn_workspace_bytes(const fastkv_shape* shape, size_t* bytes) {
+  int rc = check_shape(shape, false);
+  if (rc) return rc;
+  if (bytes == nullptr) return fail(FASTKV_ERR_INVALID_ARG, "bytes is NULL");
+  *bytes = round_up(decode_workspace_bytes(shape->batch, shape->n_kv_heads, shape->n_q_heads / shape->n_kv_heads,
+                                           shape->head_dim), 256);
+  return FASTKV_OK;
+}
+
+int fastkv_decode_attn(const fastkv_shape* shape, const void* q, const void* k_cache, const void* v_cache,
+                       const fastkv_budget* kv, float* out, float* lse, void* workspace, size_t workspace_bytes,
+                       void* stream_) {
+  int rc = check_shape(shape, false);
+  if (rc) return rc;
+  const fastkv_shape& s = *shape;
+  const int G = s.n_q_heads / s.n_kv_heads;
+  if (!q || !k_cache || !v_cache || !out) return fail(FASTKV_ERR_INVALID_ARG, "decode_attn: q, k_cache, v_cache and out are required");
+  if ((rc = check_budget(shape, kv, "decode_attn"))) return rc;
+  if (s.head_dim != 64 && s.head_dim != 128) return fail(FASTKV_ERR_UNSUPPORTED, "decode_attn: head_dim must be 64 or 128");
+  if (G > 8) return fail(FASTKV_ERR_UNSUPPORTED, "decode_attn: more than 8 query heads per KV head is not built");
+  if (reinterpret_cast<uintptr_t>(k_cache) % 16 || reinterpret_cast<uintptr_t>(v_cache) % 16)
+    return fail(FASTKV_ERR_UNSUPPORTED, "decode_attn: the caches must be 16-byte aligned");
+  if (!(s.softmax_scale >= 0.0f) || std::isinf(s.softmax_scale)) return fail(FASTKV_ERR_INVALID_ARG, "softmax_scale must be finite and >= 0");
+  const size_t need = round_up(decode_workspace_bytes(s.batch, s.n_kv_heads, G, s.head_dim), 256);
+  if ((rc = check_workspace(workspace, workspace_bytes, need))) return rc;
+  if ((rc = check_device())) return rc;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  const size_t parts = static_cast<size_t>(s.batch) * s.n_kv_heads * kDecodeMaxSplits * G;
+  DecodeParams p;
+  p.q = static_cast<const uint16_t*>(q); p.k_cache = k_cache; p.v_cache = v_cache; p.ld_cache = kv->total;
+  p.cu_k = kv->cu_k; p.k_uniform = kv->k; p.n_q_heads = s.n_q_heads; p.n_kv_heads = s.n_kv_heads; p.group = G;
+  const float scale = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / std::sqrt(static_cast<float>(s.head_dim));
+  p.scale_log2 = scale * 1.4426950408889634f;
+  p.out = out; p.lse = lse;
+  p.part_ml = reinterpret_cast<float2*>(ws + sizeof(WorkspaceHeader));
+  p.part_o = reinterpret_cast<float*>(ws + sizeof(WorkspaceHeader) + round_up(parts * sizeof(float2), 256));
+  p.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+  const int k_max = kv->cu_k ? (kv->total < s.max_len ? kv->total : s.max_len) : kv->k;
+  cudaError_t e = launch_decode_attn(p, s.head_dim, s.batch, k_max, static_cast<cudaStream_t>(stream_));
+  if (e != cudaSuccess) return cuda_fail(e, "decode_attn_kernel launch");
+  g_launches += 2;
   return FASTKV_OK;
 }
 

@@ -38,6 +38,7 @@ enum Site : int {
   SITE_FUSED_P2_DONE = 18,
   SITE_COMPACT_INDEX = 16,
   SITE_COMPACT_WAIT = 19,
+  SITE_DECODE_WAIT = 20,
   SITE_SELECT_BUDGET = 17,
 };
 

@@ -1,0 +1,29 @@
+// Parameter block and launcher of the decode-time attention over the compact cache (see decode_attn.cu).
+#pragma once
+
+#include "common.cuh"
+
+namespace fastkv {
+
+constexpr int kDecodeMaxSplits = 64;
+
+struct DecodeParams {
+  const uint16_t* q;          // [B][Hq][d] bf16 bits: one new query token per sequence
+  const void* k_cache;        // [Hkv][ld_cache][d] bf16, sequence b at rows cu_k[b] .. (or b * k_uniform ..)
+  const void* v_cache;
+  long long ld_cache;         // kept entries summed over the batch (rows per head)
+  const int* cu_k;            // device, may be null (then k_uniform)
+  int k_uniform;
+  int n_q_heads, n_kv_heads, group;
+  float scale_log2;           // softmax scale times log2(e)
+  float* out;                 // [B][Hq][d] fp32
+  float* lse;                 // [B][Hq] natural-log sum of exponentials, may be null
+  float2* part_ml;            // [B][Hkv][splits][G] per-split (max, sum) in log2 units
+  float* part_o;              // [B][Hkv][splits][G][d] per-split unnormalised outputs
+  WorkspaceHeader* hdr;
+};
+
+size_t decode_workspace_bytes(int batch, int n_kv_heads, int group, int head_dim);
+cudaError_t launch_decode_attn(DecodeParams& p, int head_dim, int batch, int k_max, cudaStream_t stream);
+
+}  // namespace fastkv
