@@ -61,7 +61,7 @@ typedef struct fastkv_shape {
   int32_t n_kv_heads;
   int32_t head_dim;         /* 64 or 128                                                      */
   int32_t hidden_dim;       /* multiple of 8; only used by fastkv_compact                     */
-  int32_t window;           /* w = N_obs (paper: 8); G*w <= 64                                */
+  int32_t window;           /* w = N_obs (paper: 8); fastkv_score needs G*w <= 64             */
   int32_t pool_kernel;      /* odd, 1..63 (paper: 7)                                          */
   int32_t pool_mode;        /* FASTKV_POOL_AVG | FASTKV_POOL_MAX                              */
   int32_t agg_order;        /* FASTKV_GROUP_THEN_POOL: pool the group-summed score;
@@ -95,7 +95,13 @@ typedef struct fastkv_budget {
   const int32_t* cu_k;
 } fastkv_budget;
 
-/* Bytes of workspace needed by the calls below for this shape (a multiple of 256). */
+/*
+ * Bytes of workspace the calls below need for this shape (a multiple of 256): what the scoring
+ * kernel that fastkv_score will pick for the shape uses -- per-phase counters, per-CTA softmax
+ * statistics and one un-pooled fp32 score row per KV head (per query head with
+ * FASTKV_POOL_THEN_GROUP), about 4.5 MB at 131072 tokens of the Llama-3.1-8B head shape -- plus the
+ * 256-byte header with the device status word.  The other calls only use the header.
+ */
 int fastkv_workspace_bytes(const fastkv_shape* shape, size_t* bytes);
 
 /*
@@ -199,19 +205,56 @@ int fastkv_layer_host(const fastkv_shape* shape, int32_t k_kv, int32_t k_tsp, co
  * memory of the scoring kernels held in a fixed 16 MiB device array inside the library (so
  * every GPU that loads the library carries those 16 MiB until the process exits).  It calls no
  * cudaMalloc, cudaFree or other allocating routine.
- *   - Limit: fastkv_workspace_bytes(shape) must be <= 16 MiB (Llama-3.1-8B head shape: up to
- *     16 000 tokens per call); larger shapes return FASTKV_ERR_WORKSPACE and launch nothing.
+ *   - Limit: fastkv_workspace_bytes(shape) must be <= 16 MiB (Llama-3.1-8B head shape: about
+ *     500 000 tokens per call); larger shapes return FASTKV_ERR_WORKSPACE and launch nothing.
  *   - The first call on each device looks up the array's device address (the device must be
  *     current); make that first call before starting any stream capture.
  *   - All calls on a device share the one array, which keeps the previous call's contents; the
  *     words that must start at zero are cleared on `stream` by every call.  Two calls whose
  *     GPU work overlaps (different streams, no ordering) race on it: serialise them.
- *   - The device status word lives inside the array and is not exposed; waits on the device
- *     stay bounded as in fastkv_score.
+ *   - The device status word lives inside the array; fastkv_score_static_status reads it.
+ *     Waits on the device stay bounded as in fastkv_score.
  * q, k, scores_kv, scores_tsp, stream: as for fastkv_score.
  */
 int fastkv_score_static(const fastkv_shape* shape, const void* q, const void* k, float* scores_kv,
                         float* scores_tsp, void* stream);
+/*
+ * fastkv_device_status for the built-in array of the current device (no counterpart in the paper):
+ * synchronises `stream`, then copies the status word and site left by the last fastkv_score_static
+ * call on this device to the HOST integers.  Allocates nothing.  FASTKV_ERR_INVALID_ARG if
+ * fastkv_score_static has not run on this device yet.
+ */
+int fastkv_score_static_status(void* stream, int32_t* status, int32_t* site);
+
+/*
+ * Test and tuning hooks (no counterpart in the paper).  Process-wide, not thread-safe; the
+ * defaults (all 0) are what production code wants.  Keys:
+ *   "score_path"          0 the library picks the scoring kernel by shape; 1 two kernels with
+ *                         fp32 logits buffered in the workspace; 2 persistent kernel that reads K
+ *                         a second time from L2; 3 persistent kernel that parks the logits in
+ *                         tensor memory (FASTKV_ERR_UNSUPPORTED from the scoring calls when a
+ *                         sequence is too long for it).  fastkv_workspace_bytes follows the choice.
+ *   "fused_heads"         path 2: KV heads scored side by side in one phase (0: by size)
+ *   "fused_lead"          path 2: phases the first read may lead the second (0: by size)
+ *   "wait_limit_cycles"   clock cycles a device-side wait of the scoring kernels polls before it
+ *                         gives up and raises FASTKV_ERR_DEVICE_TIMEOUT (0: about a second)
+ *   "extra_publications"  the scoring kernels' second pass waits for this many publications of
+ *                         softmax statistics beyond those that will arrive; with a short wait limit
+ *                         this makes a bounded wait run out without any fault (timeout test)
+ *   "time_kernels"        1: record a pair of CUDA events around every kernel the library launches
+ *                         (this creates events, and an event between two kernels keeps the second
+ *                         from starting under the first one's tail); read with
+ *                         fastkv_debug_kernel_time
+ * Unknown keys return FASTKV_ERR_INVALID_ARG.
+ */
+int fastkv_debug_set(const char* key, int64_t value);
+/*
+ * Sum of the device durations (HOST double, milliseconds) and number of launches recorded for one
+ * kernel class since the last query (0 scoring kernel, 1 pooling kernel, 2 selection, 3 compaction,
+ * 4 decode attention); waits for the recorded launches and forgets them.  *name receives a static
+ * string.  Any of the three outputs may be NULL.  No counterpart in the paper (measurement aid).
+ */
+int fastkv_debug_kernel_time(int32_t kernel, double* total_ms, int64_t* launches, const char** name);
 
 /* Text for a fastkv_status; static storage. */
 const char* fastkv_status_string(int status);

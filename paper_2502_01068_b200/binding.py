@@ -22,8 +22,11 @@ Q_FULL, Q_WINDOW = 0, 1
 
 EXPORTS = ["fastkv_workspace_bytes", "fastkv_score", "fastkv_select_kv", "fastkv_select_tsp", "fastkv_select",
            "fastkv_compact", "fastkv_decode_attn_workspace_bytes", "fastkv_decode_attn", "fastkv_device_status", "fastkv_layer_host_arena_bytes",
-           "fastkv_layer_host", "fastkv_score_static", "fastkv_status_string", "fastkv_last_error",
-           "fastkv_kernel_launches"]
+           "fastkv_layer_host", "fastkv_score_static", "fastkv_score_static_status", "fastkv_debug_set",
+           "fastkv_debug_kernel_time",
+           "fastkv_status_string", "fastkv_last_error", "fastkv_kernel_launches"]
+_INT_RETURNING = [n for n in EXPORTS if n not in ("fastkv_status_string", "fastkv_last_error",
+                                                  "fastkv_kernel_launches")]
 
 
 class FastKVError(RuntimeError):
@@ -83,7 +86,11 @@ def _load():
         lib.fastkv_score_static.argtypes = [ps, vp, vp, vp, vp, vp]
         lib.fastkv_decode_attn_workspace_bytes.argtypes = [ps, ctypes.POINTER(sz)]
         lib.fastkv_decode_attn.argtypes = [ps, vp, vp, vp, pb, vp, vp, vp, sz, vp]
-        for fn in EXPORTS[:12]:
+        lib.fastkv_score_static_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
+        lib.fastkv_debug_set.argtypes = [ctypes.c_char_p, ctypes.c_int64]
+        lib.fastkv_debug_kernel_time.argtypes = [ctypes.c_int32, ctypes.POINTER(ctypes.c_double),
+                                                 ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_char_p)]
+        for fn in _INT_RETURNING:
             getattr(lib, fn).restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -224,9 +231,31 @@ def fastkv_layer_host(shape: Shape, k_kv: int, k_tsp: int, q, k, v, hidden, pos_
 def fastkv_score_static(shape: Shape, q, k, scores_kv, scores_tsp, stream=None) -> None:
     """fastkv_score without a workspace argument: the scratch is a fixed 16 MiB array inside the
     library, for callers that cannot allocate device memory.  Shapes that need more raise
-    FastKVError(ERR_WORKSPACE).  Calls on one device share the array: do not overlap them."""
+    FastKVError(ERR_WORKSPACE).  Calls on one device share the array: do not overlap them.
+    fastkv_score_static_status() reads the device status word the call left behind."""
     _check(_load().fastkv_score_static(ctypes.byref(shape), _p(q), _p(k), _p(scores_kv), _p(scores_tsp),
                                        _stream(stream)), "fastkv_score_static")
+
+
+def fastkv_score_static_status(stream=None):
+    """(status, site) left by the last fastkv_score_static call on the current device."""
+    status, site = ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(_load().fastkv_score_static_status(_stream(stream), ctypes.byref(status), ctypes.byref(site)),
+           "fastkv_score_static_status")
+    return int(status.value), int(site.value)
+
+
+def fastkv_debug_set(key: str, value: int) -> None:
+    """Test and tuning hooks of the library (process-wide); see include/fastkv.h for the keys."""
+    _check(_load().fastkv_debug_set(key.encode(), int(value)), "fastkv_debug_set")
+
+
+def fastkv_debug_kernel_time(kernel: int):
+    """(name, total milliseconds, launches) recorded for one kernel class while the "time_kernels" hook was on."""
+    ms, n, name = ctypes.c_double(0.0), ctypes.c_int64(0), ctypes.c_char_p()
+    _check(_load().fastkv_debug_kernel_time(kernel, ctypes.byref(ms), ctypes.byref(n), ctypes.byref(name)),
+           "fastkv_debug_kernel_time")
+    return name.value.decode(), float(ms.value), int(n.value)
 
 
 def fastkv_status_string(status: int) -> str:

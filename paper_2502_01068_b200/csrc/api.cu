@@ -6,6 +6,8 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
+#include <vector>
 
 #include "compact.cuh"
 #include "decode_attn.cuh"
@@ -34,18 +36,64 @@ size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 int npad_for(int n_rows) { return n_rows <= 32 ? 32 : 64; }
 
+// ---- test and tuning hooks (fastkv_debug_set) ------------------------------------------------------
+enum ScorePath { PATH_AUTO = 0, PATH_BUFFERED = 1, PATH_REREAD = 2, PATH_PARKED = 3 };
+struct DebugConfig {
+  int score_path = PATH_AUTO;
+  int fused_heads = 0;              // two-pipeline kernel: KV heads side by side in a phase (0 = by size)
+  int fused_lead = 0;               // two-pipeline kernel: phases pass 1 may lead pass 2 (0 = by size)
+  long long wait_limit_cycles = 0;  // 0 = the default of about a second
+  int extra_publications = 0;       // pass 2 waits for publications that never come (timeout test)
+};
+DebugConfig g_debug;
+
+// ---- optional per-kernel timing ("time_kernels" hook): a pair of events around every launch ----------
+enum KernelId { KID_SCORE = 0, KID_POOL = 1, KID_SELECT = 2, KID_COMPACT = 3, KID_DECODE = 4, KID_COUNT = 5 };
+const char* const kKernelNames[KID_COUNT] = {"score", "pool", "select", "compact", "decode_attn"};
+struct KernelTimes {
+  bool on = false;
+  std::mutex mu;
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> ev[KID_COUNT];
+};
+KernelTimes g_times;
+
+struct TimedLaunch {          // records an event before and (in the destructor) after one kernel launch
+  int id;
+  cudaStream_t stream;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  TimedLaunch(int id_, cudaStream_t s) : id(id_), stream(s) {
+    if (!g_times.on) return;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) { e0 = e1 = nullptr; return; }
+    cudaEventRecord(e0, stream);
+  }
+  ~TimedLaunch() {
+    if (e0 == nullptr) return;
+    cudaEventRecord(e1, stream);
+    std::lock_guard<std::mutex> lock(g_times.mu);
+    g_times.ev[id].emplace_back(e0, e1);
+  }
+};
+
 // ---- workspace layout --------------------------------------------------------------------------
 struct Layout {
   int npad, tiles_per_cta, max_ranges;
   long long ld_logits;
-  size_t off_counters, off_final, off_partial, off_logits, bytes, zero_bytes;
-  // single-pass path (score_fused.cu): same header, its own carving of the rest
-  bool fused_shape_ok;        // the shape fits the tensor-memory-resident design on a full B200
+  size_t off_counters, off_final, off_partial, off_logits, b_bytes, zero_bytes;   // buffered path
+  // persistent one-HBM-pass kernels (score_parked.cu, score_fused.cu): same header, their own carving of the rest
+  bool fused_shape_ok;        // the shape is one the persistent kernels are built for
   int f_rows;                 // un-pooled rows written by pass 2 (KV heads or query heads)
   size_t f_off_counters, f_off_partial, f_off_a, f_zero_bytes, f_bytes;
+  int path;                   // the ScorePath fastkv_score takes for this shape; -1: the forced path cannot run it
+  size_t bytes;               // workspace that path needs
 };
 
 constexpr int kFusedMaxCtas = 148;      // SMs of a B200: one persistent CTA each
+
+// Tiles of the longest sequence one CTA parks per phase when `ctas` persistent CTAs share it.
+int parked_tiles_per_cta(int max_len, int ctas) {
+  const int ntiles = (max_len + 127) / 128;
+  return (ntiles + ctas - 1) / ctas;
+}
 
 Layout make_layout(const fastkv_shape& s) {
   Layout l;
@@ -70,7 +118,7 @@ Layout make_layout(const fastkv_shape& s) {
   off += round_up(sizeof(float2) * static_cast<size_t>(s.batch) * s.n_kv_heads * l.max_ranges * l.npad, 256);
   l.off_logits = off;
   off += round_up(sizeof(float) * static_cast<size_t>(s.n_kv_heads) * l.npad * l.ld_logits, 256);
-  l.bytes = off;
+  l.b_bytes = off;
 
   const int phases = s.batch * s.n_kv_heads;
   const bool per_head = s.agg_order == FASTKV_POOL_THEN_GROUP;
@@ -85,7 +133,17 @@ Layout make_layout(const fastkv_shape& s) {
   l.f_off_a = off;
   off += round_up(sizeof(float) * static_cast<size_t>(l.f_rows) * l.ld_logits, 256);
   l.f_bytes = off;
-  if (l.f_bytes > l.bytes) l.bytes = l.f_bytes;     // one size serves whichever path runs
+  // Which kernel scores this shape.  The parked kernel is the fastest while a CTA's tiles of two phases
+  // fit in its tensor-memory ring; longer sequences re-read K from L2 with the two-pipeline kernel; the
+  // buffered two-kernel path serves the remaining shapes.
+  const int per = parked_tiles_per_cta(s.max_len, kFusedMaxCtas), slots = parked_slots(l.npad);
+  switch (g_debug.score_path) {
+    case PATH_BUFFERED: l.path = PATH_BUFFERED; break;
+    case PATH_REREAD: l.path = l.fused_shape_ok ? PATH_REREAD : PATH_BUFFERED; break;
+    case PATH_PARKED: l.path = !l.fused_shape_ok ? PATH_BUFFERED : (per <= slots ? PATH_PARKED : -1); break;
+    default: l.path = !l.fused_shape_ok ? PATH_BUFFERED : (2 * per <= slots ? PATH_PARKED : PATH_REREAD); break;
+  }
+  l.bytes = l.path == PATH_BUFFERED ? l.b_bytes : l.f_bytes;
   return l;
 }
 
@@ -190,31 +248,39 @@ int encode_bf16_3d(CUtensorMap* map, const void* base, int dim, int heads, long 
 
 // Persistent CTAs the single-pass scoring kernel may use: one per SM, capped at the count the
 // workspace is carved for; 0 if the device cannot be queried or has no cooperative launch.
+// (cached per device ordinal: one process may drive several GPUs)
 int fused_grid() {
-  static int ctas = -1;
-  if (ctas < 0) {
-    int dev = 0, sms = 0, coop = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+  static int ctas[PerDeviceOnce::kMaxDevices];
+  static PerDeviceOnce known;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= PerDeviceOnce::kMaxDevices) return 0;
+  if (!known.done(dev)) {
+    int sms = 0, coop = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop)
-      ctas = 0;
+      ctas[dev] = 0;
     else
-      ctas = sms < kFusedMaxCtas ? sms : kFusedMaxCtas;
+      ctas[dev] = sms < kFusedMaxCtas ? sms : kFusedMaxCtas;
+    known.set(dev);
   }
-  return ctas;
+  return ctas[dev];
 }
 
 int check_device() {
-  static int ok = -1;
-  if (ok < 0) {
-    int dev = 0, major = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+  static int ok[PerDeviceOnce::kMaxDevices];
+  static PerDeviceOnce known;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+  if (dev < 0 || dev >= PerDeviceOnce::kMaxDevices) return fail(FASTKV_ERR_UNSUPPORTED, "device ordinal out of range");
+  if (!known.done(dev)) {
+    int major = 0;
     e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
     if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
-    ok = (major == 10) ? 1 : 0;
+    ok[dev] = (major == 10) ? 1 : 0;
+    known.set(dev);
   }
-  if (!ok) return fail(FASTKV_ERR_UNSUPPORTED, "this library is built for sm_100a (B200) only");
+  if (!ok[dev]) return fail(FASTKV_ERR_UNSUPPORTED, "this library is built for sm_100a (B200) only");
   return FASTKV_OK;
 }
 
@@ -234,7 +300,51 @@ int fastkv_workspace_bytes(const fastkv_shape* shape, size_t* bytes) {
   int rc = check_shape(shape, true);
   if (rc) return rc;
   if (bytes == nullptr) return fail(FASTKV_ERR_INVALID_ARG, "bytes is NULL");
-  *bytes = make_layout(*shape).bytes;
+  const Layout lay = make_layout(*shape);
+  if (lay.path < 0) return fail(FASTKV_ERR_UNSUPPORTED, "the forced scoring path cannot run this shape");
+  *bytes = lay.bytes;
+  return FASTKV_OK;
+}
+
+int fastkv_debug_set(const char* key, int64_t value) {
+  if (key == nullptr) return fail(FASTKV_ERR_INVALID_ARG, "debug_set: key is NULL");
+  if (!std::strcmp(key, "score_path")) {
+    if (value < PATH_AUTO || value > PATH_PARKED) return fail(FASTKV_ERR_INVALID_ARG, "debug_set: score_path is 0..3");
+    g_debug.score_path = static_cast<int>(value);
+  } else if (!std::strcmp(key, "fused_heads")) {
+    g_debug.fused_heads = static_cast<int>(value < 0 ? 0 : value);
+  } else if (!std::strcmp(key, "fused_lead")) {
+    g_debug.fused_lead = static_cast<int>(value < 0 ? 0 : value);
+  } else if (!std::strcmp(key, "wait_limit_cycles")) {
+    g_debug.wait_limit_cycles = value < 0 ? 0 : value;
+  } else if (!std::strcmp(key, "extra_publications")) {
+    g_debug.extra_publications = static_cast<int>(value < 0 ? 0 : value);
+  } else if (!std::strcmp(key, "time_kernels")) {
+    g_times.on = value != 0;
+  } else {
+    return fail(FASTKV_ERR_INVALID_ARG, "debug_set: unknown key '%s'", key);
+  }
+  return FASTKV_OK;
+}
+
+int fastkv_debug_kernel_time(int32_t kernel, double* total_ms, int64_t* launches, const char** name) {
+  if (kernel < 0 || kernel >= KID_COUNT) return fail(FASTKV_ERR_INVALID_ARG, "debug_kernel_time: kernel is 0..%d", KID_COUNT - 1);
+  std::lock_guard<std::mutex> lock(g_times.mu);
+  double ms = 0.0;
+  int64_t n = 0;
+  for (auto& pr : g_times.ev[kernel]) {
+    float t = 0.0f;
+    if (cudaEventSynchronize(pr.second) == cudaSuccess && cudaEventElapsedTime(&t, pr.first, pr.second) == cudaSuccess) {
+      ms += t;
+      ++n;
+    }
+    cudaEventDestroy(pr.first);
+    cudaEventDestroy(pr.second);
+  }
+  g_times.ev[kernel].clear();
+  if (total_ms) *total_ms = ms;
+  if (launches) *launches = n;
+  if (name) *name = kKernelNames[kernel];
   return FASTKV_OK;
 }
 
@@ -245,6 +355,7 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
   if (q == nullptr || k == nullptr || scores_kv == nullptr)
     return fail(FASTKV_ERR_INVALID_ARG, "q, k and scores_kv are required");
   const Layout lay = make_layout(*shape);
+  if (lay.path < 0) return fail(FASTKV_ERR_UNSUPPORTED, "the forced scoring path cannot run this shape");
   if ((rc = check_workspace(workspace, workspace_bytes, lay.bytes))) return rc;
   if ((rc = check_device())) return rc;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -264,12 +375,14 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
   const float scale = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / std::sqrt(static_cast<float>(s.head_dim));
   const float scale_log2 = scale * 1.4426950408889634f;
   WorkspaceHeader* hdr = reinterpret_cast<WorkspaceHeader*>(ws);
-  const int ctas = fused_grid();
-  const char* force = std::getenv("FASTKV_SCORE_PATH");        // "buffered" forces the two-pass path
-  const bool fused = lay.fused_shape_ok && ctas > 0 && !(force && std::strcmp(force, "buffered") == 0);
   cudaError_t e;
-  if (fused) {
-    // ---- one HBM pass over K: persistent two-pipeline kernel ----
+  if (lay.path != PATH_BUFFERED) {
+    // ---- one HBM pass over K: persistent kernel, one CTA per SM ----
+    const int ctas = fused_grid();
+    if (ctas <= 0) return fail(FASTKV_ERR_UNSUPPORTED, "the device offers no cooperative launch");
+    const bool parked = lay.path == PATH_PARKED;
+    if (parked && parked_tiles_per_cta(s.max_len, ctas) > parked_slots(lay.npad))
+      return fail(FASTKV_ERR_UNSUPPORTED, "this device has too few SMs to park a phase of this length");
     e = cudaMemsetAsync(ws, 0, lay.f_zero_bytes, stream);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace header)");
     FusedParams fp;
@@ -281,22 +394,27 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
     // A phase is sized to about one head of a 128K-token sequence (33.5 MB of K): shorter sequences put several
     // heads side by side in a phase, so that there are fewer grid-wide dependencies per byte.  Pass 1 may lead pass 2
     // by as many phases as keep about 110 MB of K between the two reads: that is what stays in the 126 MB L2.
-    const char* hpp = std::getenv("FASTKV_FUSED_HEADS");     // tuning knobs
-    const char* lead = std::getenv("FASTKV_FUSED_LEAD");
-    fp.heads_per_phase = hpp ? std::atoi(hpp) : 0;
+    fp.heads_per_phase = g_debug.fused_heads;
     fp.phase_bytes = 35000000;
     fp.head_bytes = static_cast<long long>(s.head_dim) * 2;
     double longest_phase = static_cast<double>(s.max_len) * s.head_dim * 2.0;     // bytes of the largest phase
     const double hp_longest = fp.heads_per_phase > 0 ? fp.heads_per_phase : fp.phase_bytes / longest_phase;
     if (hp_longest >= 1.0) longest_phase *= static_cast<int>(hp_longest < s.n_kv_heads ? hp_longest : s.n_kv_heads);
-    fp.max_lead = lead ? std::atoi(lead) : static_cast<int>(110e6 / longest_phase);
+    fp.max_lead = g_debug.fused_lead > 0 ? g_debug.fused_lead : static_cast<int>(110e6 / longest_phase);
     if (fp.max_lead > (1 << 20)) fp.max_lead = 1 << 20;
     if (fp.max_lead < 2) fp.max_lead = 2;
     fp.partial = reinterpret_cast<float2*>(ws + lay.f_off_partial);
     fp.counters = reinterpret_cast<int*>(ws + lay.f_off_counters);
     fp.hdr = hdr;
-    e = launch_score_fused(s.head_dim, lay.npad, tmap_k, tmap_q, fp, ctas, stream);
-    if (e != cudaSuccess) return cuda_fail(e, "score_fused_kernel launch");
+    fp.max_len = s.max_len;
+    fp.wait_limit = g_debug.wait_limit_cycles > 0 ? g_debug.wait_limit_cycles : kWaitLimitCycles;
+    fp.extra_publications = g_debug.extra_publications;
+    {
+      TimedLaunch timed(KID_SCORE, stream);
+      e = parked ? launch_score_parked(s.head_dim, lay.npad, tmap_k, tmap_q, fp, ctas, stream)
+                 : launch_score_fused(s.head_dim, lay.npad, tmap_k, tmap_q, fp, ctas, stream);
+    }
+    if (e != cudaSuccess) return cuda_fail(e, parked ? "score_parked_kernel launch" : "score_fused_kernel launch");
     ++g_launches;
     PoolRowsParams rp;
     rp.total_len = s.total_len; rp.n_kv_heads = s.n_kv_heads; rp.group = G; rp.window = s.window;
@@ -305,7 +423,10 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
     rp.scores_kv = scores_kv; rp.ld_scores = s.total_len; rp.scores_tsp = scores_tsp;
     if (sizeof(float) * static_cast<size_t>(lay.f_rows) * (kPoolKeys + s.pool_kernel) > 200 * 1024)
       return fail(FASTKV_ERR_UNSUPPORTED, "heads x pool halo do not fit the pooling kernel's shared memory");
-    e = launch_pool_rows(rp, s.max_len, s.batch, stream);
+    {
+      TimedLaunch timed(KID_POOL, stream);
+      e = launch_pool_rows(rp, s.max_len, s.batch, stream);
+    }
     if (e != cudaSuccess) return cuda_fail(e, "pool_rows_kernel launch");
     ++g_launches;
     return FASTKV_OK;
@@ -328,7 +449,10 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
   sp.counters = reinterpret_cast<int*>(ws + lay.off_counters);
   sp.hdr = hdr;
   dim3 grid(s.n_kv_heads, lay.max_ranges, s.batch);
-  e = launch_score_logits(s.head_dim, lay.npad, tmap_k, tmap_q, sp, grid, stream);
+  {
+    TimedLaunch timed(KID_SCORE, stream);
+    e = launch_score_logits(s.head_dim, lay.npad, tmap_k, tmap_q, sp, grid, stream);
+  }
   if (e != cudaSuccess) return cuda_fail(e, "score_logits_kernel launch");
   ++g_launches;
 
@@ -340,7 +464,10 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
   pp.scores_tsp = scores_tsp;
   if (score_pool_smem_bytes(pp) > 200 * 1024)
     return fail(FASTKV_ERR_UNSUPPORTED, "heads x pool halo do not fit the pooling kernel's shared memory");
-  e = launch_score_pool(pp, s.max_len, s.batch, stream);
+  {
+    TimedLaunch timed(KID_POOL, stream);
+    e = launch_score_pool(pp, s.max_len, s.batch, stream);
+  }
   if (e != cudaSuccess) return cuda_fail(e, "score_pool_kernel launch");
   ++g_launches;
   return FASTKV_OK;
@@ -363,7 +490,11 @@ static int launch_select_sets(const fastkv_shape* shape, SelectParams& p, void* 
   if ((rc = check_device())) return rc;
   p.cu_seqlens = shape->cu_seqlens; p.total_len = shape->total_len; p.window = shape->window;
   p.force_window = shape->force_window; p.hdr = static_cast<WorkspaceHeader*>(workspace);
-  cudaError_t e = launch_select(p, shape->batch, shape->max_len, static_cast<cudaStream_t>(stream_));
+  cudaError_t e;
+  {
+    TimedLaunch timed(KID_SELECT, static_cast<cudaStream_t>(stream_));
+    e = launch_select(p, shape->batch, shape->max_len, static_cast<cudaStream_t>(stream_));
+  }
   if (e != cudaSuccess) return cuda_fail(e, "select_topk_kernel launch");
   ++g_launches;
   return FASTKV_OK;
@@ -453,7 +584,11 @@ int fastkv_compact(const fastkv_shape* shape, const int32_t* idx_kv, const fastk
   cp.n_jobs = n;
   if (n == 0) return FASTKV_OK;
   if ((rc = check_device())) return rc;
-  cudaError_t e = launch_compact(cp, static_cast<cudaStream_t>(stream_));
+  cudaError_t e;
+  {
+    TimedLaunch timed(KID_COMPACT, static_cast<cudaStream_t>(stream_));
+    e = launch_compact(cp, static_cast<cudaStream_t>(stream_));
+  }
   if (e != cudaSuccess) return cuda_fail(e, "compact_rows_kernel launch");
   ++g_launches;
   return FASTKV_OK;
@@ -497,7 +632,11 @@ int fastkv_decode_attn(const fastkv_shape* shape, const void* q, const void* k_c
   p.part_o = reinterpret_cast<float*>(ws + sizeof(WorkspaceHeader) + round_up(parts * sizeof(float2), 256));
   p.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
   const int k_max = kv->cu_k ? (kv->total < s.max_len ? kv->total : s.max_len) : kv->k;
-  cudaError_t e = launch_decode_attn(p, s.head_dim, s.batch, k_max, static_cast<cudaStream_t>(stream_));
+  cudaError_t e;
+  {
+    TimedLaunch timed(KID_DECODE, static_cast<cudaStream_t>(stream_));
+    e = launch_decode_attn(p, s.head_dim, s.batch, k_max, static_cast<cudaStream_t>(stream_));
+  }
   if (e != cudaSuccess) return cuda_fail(e, "decode_attn_kernel launch");
   g_launches += 2;
   return FASTKV_OK;
@@ -519,7 +658,7 @@ int fastkv_device_status(const void* workspace, void* stream, int32_t* status, i
 namespace {
 struct Arena {
   size_t q, k, v, hidden, pos, cu, scores_kv, scores_tsp, idx_kv, idx_tsp, k_out, v_out, hidden_out, pos_out, ws;
-  size_t q_bytes, kv_bytes, hidden_bytes, ws_bytes, bytes;
+  size_t q_bytes, k_bytes, v_bytes, hidden_bytes, ws_bytes, bytes;
 };
 Arena make_arena(const fastkv_shape& s, int k_kv, int k_tsp) {
   Arena a;
@@ -527,9 +666,10 @@ Arena make_arena(const fastkv_shape& s, int k_kv, int k_tsp) {
   auto take = [&](size_t n) { size_t o = off; off += round_up(n, 256); return o; };
   const size_t q_rows = s.q_layout == FASTKV_Q_WINDOW ? static_cast<size_t>(s.batch) * s.window : s.total_len;
   a.q_bytes = q_rows * s.q_stride_tok * 2;
-  a.kv_bytes = static_cast<size_t>(s.total_len) * s.k_stride_tok * 2;
+  a.k_bytes = static_cast<size_t>(s.total_len) * s.k_stride_tok * 2;
+  a.v_bytes = static_cast<size_t>(s.total_len) * s.v_stride_tok * 2;
   a.hidden_bytes = static_cast<size_t>(s.total_len) * s.hidden_stride_tok * 2;
-  a.q = take(a.q_bytes); a.k = take(a.kv_bytes); a.v = take(a.kv_bytes);
+  a.q = take(a.q_bytes); a.k = take(a.k_bytes); a.v = take(a.v_bytes);
   a.hidden = take(k_tsp ? a.hidden_bytes : 0); a.pos = take(k_tsp ? 4 * static_cast<size_t>(s.total_len) : 0);
   a.cu = take(4 * (static_cast<size_t>(s.batch) + 1));
   a.scores_kv = take(4 * static_cast<size_t>(s.n_kv_heads) * s.total_len);
@@ -575,8 +715,8 @@ int fastkv_layer_host(const fastkv_shape* shape, int32_t k_kv, int32_t k_tsp, co
 #define FASTKV_COPY(dst, src, n, kind)                                             \
   if ((n) && (e = cudaMemcpyAsync(dst, src, n, kind, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync")
   FASTKV_COPY(d + a.q, q, a.q_bytes, cudaMemcpyHostToDevice);
-  FASTKV_COPY(d + a.k, k, a.kv_bytes, cudaMemcpyHostToDevice);
-  FASTKV_COPY(d + a.v, v, a.kv_bytes, cudaMemcpyHostToDevice);
+  FASTKV_COPY(d + a.k, k, a.k_bytes, cudaMemcpyHostToDevice);
+  FASTKV_COPY(d + a.v, v, a.v_bytes, cudaMemcpyHostToDevice);
   if (k_tsp) {
     FASTKV_COPY(d + a.hidden, hidden, a.hidden_bytes, cudaMemcpyHostToDevice);
     FASTKV_COPY(d + a.pos, pos_ids, 4 * static_cast<size_t>(s.total_len), cudaMemcpyHostToDevice);

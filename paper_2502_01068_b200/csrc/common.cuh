@@ -40,6 +40,11 @@ enum Site : int {
   SITE_COMPACT_WAIT = 19,
   SITE_DECODE_WAIT = 20,
   SITE_SELECT_BUDGET = 17,
+  SITE_PARKED_RING = 21,
+  SITE_PARKED_DRAIN = 22,
+  SITE_PARKED_REF = 23,
+  SITE_PARKED_STATS = 24,
+  SITE_PARKED_NORM = 25,
 };
 
 // Records `text` as the calling thread's last error (see fastkv_last_error) and returns `status`.
@@ -86,23 +91,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Every wait in these kernels is bounded: after about a second of polling the waiter records
-// where it gave up, raises the CTA-wide abort flag and returns false; callers leave their loop
-// and fall through to the common exit, so the kernel always terminates and the context stays
-// usable.  `abort_flag` lives in shared memory.
+// Every wait in these kernels is bounded: after `limit` cycles of polling (about a second by default)
+// the waiter records where it gave up, raises the CTA-wide abort flag and returns false; a waiter that
+// finds the flag already raised returns false at once.  Callers then run through the rest of their
+// loops without waiting or computing, so the kernel always terminates and the context stays usable.
+// `abort_flag` lives in shared memory.
 constexpr long long kWaitLimitCycles = 1ll << 31;
 
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity,
                                                   volatile int* abort_flag, WorkspaceHeader* hdr,
-                                                  int site) {
+                                                  int site, long long limit = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
+  if (*abort_flag) return false;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 0xFFu) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit) {
         *abort_flag = 1;
         raise_status(hdr, FASTKV_ERR_DEVICE_TIMEOUT, site);
         return false;
@@ -111,7 +118,33 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
   }
 }
 
-// ---- TMA (cp.async.bulk.tensor), plain loads only: no cluster multicast anywhere -------------
+// The wait a role uses for its own copies or contractions still in flight before it leaves: bounded
+// like every other wait, but it does not give up just because the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity, WorkspaceHeader* hdr, int site,
+                                                long long limit = kWaitLimitCycles) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 0xFFu) == 0 && clock64() - t0 > limit) {
+      raise_status(hdr, FASTKV_ERR_DEVICE_TIMEOUT, site);
+      return false;
+    }
+  }
+}
+
+// ---- global-memory publication between CTAs ---------------------------------------------------
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void red_release_add(int* p, int v) {
+  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// ---- TMA (cp.async.bulk.tensor): plain per-CTA loads only --------------------------------------
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
@@ -244,6 +277,20 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, float (&v)[16]) {
       : "memory");
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// 16 registers per thread -> 32 lanes x 16 consecutive fp32 columns of tensor memory
+__device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const float (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])),
+        "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])),
+        "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+        "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15]))
+      : "memory");
 }
 
 // 8-column variants (used where registers are scarce)
@@ -391,6 +438,15 @@ __device__ __forceinline__ float2 merge_partials(const float2* part, int npad, i
   }
   return make_float2(m, l);
 }
+
+// "Done once per device" flag for launch attributes (they are per device, and one process may
+// drive several): indexed by the device ordinal.
+struct PerDeviceOnce {
+  static constexpr int kMaxDevices = 64;
+  unsigned char flag[kMaxDevices] = {};
+  bool done(int dev) const { return dev >= 0 && dev < kMaxDevices && flag[dev] != 0; }
+  void set(int dev) { if (dev >= 0 && dev < kMaxDevices) flag[dev] = 1; }
+};
 
 // Launch configuration shared by the kernels that follow another kernel of the step.
 inline void fill_pdl_attribute(cudaLaunchAttribute* attr) {

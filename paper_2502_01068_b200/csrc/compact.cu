@@ -186,11 +186,11 @@ cudaError_t launch_compact(CompactParams& p, cudaStream_t stream) {
   }
   p.total_chunks = first;
   if (first == 0) return cudaSuccess;
-  static bool configured = false;
-  if (!configured) {
+  static PerDeviceOnce configured;        // launch attributes are per device
+  if (!configured.done(dev)) {
     cudaError_t e = cudaFuncSetAttribute(compact_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCompactSmem);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured.set(dev);
   }
   long long blocks = (first + kCompactWarps - 1) / kCompactWarps;
   if (blocks > sms) blocks = sms;

@@ -248,22 +248,25 @@ size_t decode_workspace_bytes(int batch, int n_kv_heads, int group, int head_dim
 template <int D>
 static cudaError_t launch_decode_t(DecodeParams& p, int batch, int k_max, cudaStream_t stream) {
   constexpr int kSmem = 2 * kDecStages * kDecChunk * D * 2 + kMaxGroup * D * 4 + 2 * kDecChunk * kMaxGroup * 4 + 4 * kMaxGroup * 4 + 128;
-  static bool configured = false;
-  if (!configured) {
+  // launch attributes and occupancy are per device: cached by device ordinal
+  static PerDeviceOnce configured;
+  static int capacity_of[PerDeviceOnce::kMaxDevices];
+  int dev = 0;
+  cudaError_t e0 = cudaGetDevice(&dev);
+  if (e0 != cudaSuccess) return e0;
+  if (dev < 0 || dev >= PerDeviceOnce::kMaxDevices) return cudaErrorInvalidDevice;
+  if (!configured.done(dev)) {
     cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
-    configured = true;
-  }
-  // one wave: as many splits as keep every CTA resident at once, at least one chunk per split
-  static int capacity = 0;
-  if (capacity == 0) {
-    int dev = 0, sms = 148, per_sm = 1;
-    cudaGetDevice(&dev);
+    // one wave: as many splits as keep every CTA resident at once, at least one chunk per split
+    int sms = 148, per_sm = 1;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_attn_kernel<D>, kDecThreads, kSmem) != cudaSuccess || per_sm < 1)
       per_sm = 1;
-    capacity = sms * per_sm;
+    capacity_of[dev] = sms * per_sm;
+    configured.set(dev);
   }
+  const int capacity = capacity_of[dev];
   int splits = capacity / (batch * p.n_kv_heads);
   const int chunks = (k_max + kDecChunk - 1) / kDecChunk;
   if (splits > chunks) splits = chunks;

@@ -339,12 +339,15 @@ template <int D, int NPAD>
 static cudaError_t launch_logits_t(const CUtensorMap& tk, const CUtensorMap& tq, const ScoreParams& p,
                                    dim3 grid, cudaStream_t stream) {
   using Cfg = ScoreCfg<D, NPAD>;
-  static bool configured = false;   // idempotent attribute; a race only repeats the call
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(score_logits_kernel<D, NPAD>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+  static PerDeviceOnce configured;   // per device; idempotent attribute, a race only repeats the call
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (!configured.done(dev)) {
+    e = cudaFuncSetAttribute(score_logits_kernel<D, NPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Cfg::kSmemBytes);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured.set(dev);
   }
   score_logits_kernel<D, NPAD><<<grid, kScoreThreads, Cfg::kSmemBytes, stream>>>(tk, tq, p);
   return cudaGetLastError();
@@ -367,12 +370,10 @@ size_t score_pool_smem_bytes(const PoolParams& p) {
 
 cudaError_t launch_score_pool(const PoolParams& p, int max_len, int batch, cudaStream_t stream) {
   const size_t smem = score_pool_smem_bytes(p);
-  static size_t configured = 48 * 1024;
-  if (smem > configured) {
+  if (smem > 48 * 1024) {          // rare (many heads, wide pooling window): opt in on every such launch
     cudaError_t e = cudaFuncSetAttribute(score_pool_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(smem));
     if (e != cudaSuccess) return e;
-    configured = smem;
   }
   dim3 grid((max_len + kPoolKeys - 1) / kPoolKeys, batch);
   score_pool_kernel<<<grid, kPoolThreads, smem, stream>>>(p);

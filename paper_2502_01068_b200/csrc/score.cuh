@@ -54,6 +54,9 @@ struct FusedParams {
   float2* partial;            // [phases][CTAs][NPAD]
   int* counters;              // [phases] CTAs that published their statistics (zero before launch)
   WorkspaceHeader* hdr;
+  int max_len;                // longest sequence of the batch (host knowledge)
+  long long wait_limit;       // cycles a device-side wait may poll before it gives up
+  int extra_publications;     // test hook: pass 2 waits for this many publications that never come
 };
 
 struct PoolRowsParams {
@@ -69,6 +72,10 @@ struct PoolRowsParams {
 
 cudaError_t launch_score_fused(int head_dim, int npad, const CUtensorMap& tmap_k, const CUtensorMap& tmap_q,
                                const FusedParams& p, int grid, cudaStream_t stream);
+// one pass over K, one contraction per tile, logits parked in tensor memory (score_parked.cu)
+cudaError_t launch_score_parked(int head_dim, int npad, const CUtensorMap& tmap_k, const CUtensorMap& tmap_q,
+                                const FusedParams& p, int grid, cudaStream_t stream);
+int parked_slots(int npad);   // tiles of one phase a CTA can park: its tiles per phase must not exceed this
 cudaError_t launch_pool_rows(const PoolRowsParams& p, int max_len, int batch, cudaStream_t stream);
 
 cudaError_t launch_score_logits(int head_dim, int npad, const CUtensorMap& tmap_k,

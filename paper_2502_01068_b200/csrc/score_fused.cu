@@ -50,6 +50,7 @@ struct FusedBarriers {
   uint64_t full2[4], empty2[4];
   uint64_t q1_full[2], q1_empty[2], q2_full[2], q2_empty[2];
   uint64_t acc1_full[kAcc], acc1_empty[kAcc], acc2_full[kAcc], acc2_empty[kAcc];
+  uint64_t mma_done[2];
   uint32_t tmem_base;
   int abort_flag;
   int p1_done;                 // phases (this CTA took part in) whose pass 1 is published
@@ -61,23 +62,15 @@ template <int ID>
 __device__ __forceinline__ void group_sync() { asm volatile("bar.sync %0, %1;" ::"n"(ID), "n"(kGroupWarps * 32) : "memory"); }
 
 
-__device__ __forceinline__ int ld_acquire(const int* p) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void red_release_add(int* p, int v) {
-  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-
 // Bounded wait until *flag (shared memory, written by another warp of the CTA) reaches `target`.
 __device__ __forceinline__ bool wait_smem_counter(volatile int* flag, int target, volatile int* abort_flag,
-                                                  WorkspaceHeader* hdr, int site) {
+                                                  WorkspaceHeader* hdr, int site, long long limit) {
   if (*flag >= target) return true;
+  if (*abort_flag) return false;
   const long long t0 = clock64();
   unsigned spins = 0;
   while (*flag < target) {
-    if ((++spins & 0x3Fu) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) {
+    if ((++spins & 0x3Fu) == 0 && (*abort_flag || clock64() - t0 > limit)) {
       *abort_flag = 1;
       raise_status(hdr, FASTKV_ERR_DEVICE_TIMEOUT, site);
       return false;
@@ -161,6 +154,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, ncta = gridDim.x;
+  const long long limit = p.wait_limit;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::kStages1; ++s) { mbar_init(&bars->full1[s], 1); mbar_init(&bars->empty1[s], 1); }
@@ -173,6 +167,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       mbar_init(&bars->acc1_full[i], 1); mbar_init(&bars->acc1_empty[i], kGroupWarps);   // every warp of the group
       mbar_init(&bars->acc2_full[i], 1); mbar_init(&bars->acc2_empty[i], 4);             // the four warps of one set
     }
+    mbar_init(&bars->mma_done[0], 1);
+    mbar_init(&bars->mma_done[1], 1);
     bars->abort_flag = 0;
     bars->p1_done = 0;
     bars->p2_done = 0;
@@ -207,7 +203,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       uint64_t* const q_empty = second ? bars->q2_empty : bars->q1_empty;
       const int stages = second ? Cfg::kStages2 : Cfg::kStages1;
       const int nq = second ? 1 : 2;                     // Q buffers of the pipeline
-      int it = 0, u = 0;
+      int it = 0, u = 0, uq = 0;
       bool ok = true;
       PhaseIter pit = {0, 0};
       PhaseWork w;
@@ -215,19 +211,20 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         if (w.n == 0) continue;
         // pipeline 2 re-reads what pipeline 1 of this CTA has finished with; pipeline 1 stays close
         // enough ahead for those tiles to be still in L2
-        if (second) ok = wait_smem_counter(&bars->p1_done, u + 1, abort_flag, p.hdr, SITE_FUSED_P1_DONE);
-        else if (u >= p.max_lead) ok = wait_smem_counter(&bars->p2_done, u - p.max_lead + 1, abort_flag, p.hdr, SITE_FUSED_P2_DONE);
+        if (second) ok = wait_smem_counter(&bars->p1_done, u + 1, abort_flag, p.hdr, SITE_FUSED_P1_DONE, limit);
+        else if (u >= p.max_lead) ok = wait_smem_counter(&bars->p2_done, u - p.max_lead + 1, abort_flag, p.hdr, SITE_FUSED_P2_DONE, limit);
         const int h = u % nq;
-        if (ok && u >= nq) ok = mbar_wait_bounded(&q_empty[h], ((u / nq) - 1) & 1, abort_flag, p.hdr, SITE_FUSED_Q_EMPTY);
+        if (ok && u >= nq) ok = mbar_wait_bounded(&q_empty[h], ((u / nq) - 1) & 1, abort_flag, p.hdr, SITE_FUSED_Q_EMPTY, limit);
         if (!ok) break;
         const int q_row0 = (p.q_layout == FASTKV_Q_WINDOW) ? w.b * p.window : w.row0 + w.L - p.window;
         mbar_arrive_expect_tx(&q_full[h], Cfg::KH * p.n_rows * 128);
         for (int c = 0; c < Cfg::KH; ++c)
           tma_load_3d(qbuf + h * Cfg::kQBytes + c * NPAD * 128, &tmap_q, &q_full[h], c * 64, w.g * p.group, q_row0,
                       pol_q);
+        ++uq;
         for (int i = 0; i < w.n; ++i, ++it) {
           const int s = it % stages;
-          ok = mbar_wait_bounded(&empty[s], ((it / stages) & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_EMPTY);
+          ok = mbar_wait_bounded(&empty[s], ((it / stages) & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_EMPTY, limit);
           if (!ok) break;
           mbar_arrive_expect_tx(&full[s], Cfg::kStageBytes);
           for (int c = 0; c < Cfg::KH; ++c)
@@ -235,6 +232,16 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                         w.row0 + (w.t0 + i) * kTileKeys, pol_k);
         }
         ++u;
+      }
+      // No copy may still be writing this CTA's shared memory when the CTA ends: wait for the last
+      // load of every stage and query buffer, whatever the abort flag says.
+      for (int s = 0; s < stages && s < it; ++s) {
+        const int last = it - 1 - ((it - 1 - s) % stages);
+        mbar_wait_drain(&full[s], (last / stages) & 1, p.hdr, SITE_PARKED_DRAIN, limit);
+      }
+      for (int h = 0; h < nq && h < uq; ++h) {
+        const int last = uq - 1 - ((uq - 1 - h) % nq);
+        mbar_wait_drain(&q_full[h], (last / nq) & 1, p.hdr, SITE_PARKED_DRAIN, limit);
       }
     }
   } else if (warp == 1 || warp == 3) {
@@ -260,13 +267,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       while (ok && next_phase(p, pit, cta, ncta, w)) {
         if (w.n == 0) continue;
         const int h = u % nq;
-        ok = mbar_wait_bounded(&q_full[h], (u / nq) & 1, abort_flag, p.hdr, SITE_FUSED_Q_FULL);
+        ok = mbar_wait_bounded(&q_full[h], (u / nq) & 1, abort_flag, p.hdr, SITE_FUSED_Q_FULL, limit);
         if (!ok) break;
         const uint32_t q_addr = smem_u32(qbuf + h * Cfg::kQBytes);
         for (int i = 0; i < w.n; ++i, ++it) {
           const int s = it % stages, a = it % kAcc;
-          ok = mbar_wait_bounded(&acc_empty[a], ((it / kAcc) & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_ACC_FREE) &&
-               mbar_wait_bounded(&full[s], (it / stages) & 1, abort_flag, p.hdr, SITE_FUSED_FULL);
+          ok = mbar_wait_bounded(&acc_empty[a], ((it / kAcc) & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_ACC_FREE, limit) &&
+               mbar_wait_bounded(&full[s], (it / stages) & 1, abort_flag, p.hdr, SITE_FUSED_FULL, limit);
           if (!ok) break;
           tc_fence_after_sync();
           const uint32_t k_addr = smem_u32(ring + s * Cfg::kStageBytes);
@@ -282,6 +289,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         if (ok) tc_commit(&q_empty[h]);
         ++u;
       }
+      // every contraction issued above has finished before tensor memory is released
+      if (it > 0) {
+        tc_commit(&bars->mma_done[second ? 1 : 0]);
+        mbar_wait_drain(&bars->mma_done[second ? 1 : 0], 0, p.hdr, SITE_PARKED_DRAIN, limit);
+      }
     }
   } else if (warp < kCtrlWarps + kGroupWarps) {
     // ---------------- group A: pass 1, running (max, sum of exp2) per query row; publish per phase ----------------
@@ -291,14 +303,14 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const int quarter = warp & 3, half = gw >> 2;
     const int key_in_tile = quarter * 32 + lane;
     const int at = threadIdx.x - kCtrlWarps * 32;       // 0..255 within the group
-    const int n_rows = p.n_rows, G = p.group;
+    const int n_rows = p.n_rows;
     const int col0 = half * CPW;                         // first query row of this warp
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + col0;
     int it = 0, u = 0;
     bool ok = true;
     PhaseIter pit = {0, 0};
     PhaseWork w;
-    while (ok && next_phase(p, pit, cta, ncta, w)) {
+    while (next_phase(p, pit, cta, ncta, w)) {           // an aborted CTA still walks every phase: see group_sync
       if (w.n == 0) {
         // a sequence shorter than the observation window has no defined scores: say so once
         if (w.L < p.window && cta == 0 && at == 0) raise_status(p.hdr, FASTKV_ERR_INVALID_ARG, SITE_SCORE_SHORT_SEQUENCE);
@@ -310,9 +322,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       const int win_start = w.L - p.window;
       for (int i = 0; i < w.n; ++i, ++it) {
         const int a = it % kAcc;
-        ok = mbar_wait_bounded(&bars->acc1_full[a], (it / kAcc) & 1, abort_flag, p.hdr, SITE_FUSED_ACC_FULL);
+        if (ok) ok = mbar_wait_bounded(&bars->acc1_full[a], (it / kAcc) & 1, abort_flag, p.hdr, SITE_FUSED_ACC_FULL, limit);
         ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
+        if (!ok) continue;                               // aborted: no more waiting or computing
         tc_fence_after_sync();
         const int key = (w.t0 + i) * kTileKeys + key_in_tile;
         const bool tile_unmasked = (w.t0 + i + 1) * kTileKeys <= win_start;
@@ -340,7 +352,6 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           }
         }
       }
-      if (!ok) break;
       // lanes -> warp: after the butterfly lanes r and r + 16 hold row col0 + c * 16 + r in entry c * 16
 #pragma unroll
       for (int c = 0; c < CPW / 16; ++c) {
@@ -377,16 +388,17 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     bool ok = true;
     PhaseIter pit = {0, 0};
     PhaseWork w;
-    while (ok && next_phase(p, pit, cta, ncta, w)) {
+    while (next_phase(p, pit, cta, ncta, w)) {
       if (w.n == 0) continue;
       // every CTA that owns tiles of this phase has published its statistics?
-      if (bt == 0) {
+      if (bt == 0 && !*abort_flag) {
         const int* ctr = p.counters + w.stat;
-        if (ld_acquire(ctr) < w.nact) {
+        const int target = w.nact + p.extra_publications;
+        if (ld_acquire(ctr) < target) {
           const long long t0 = clock64();
           unsigned spins = 0;
-          while (ld_acquire(ctr) < w.nact) {
-            if ((++spins & 0x3Fu) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) {
+          while (ld_acquire(ctr) < target) {
+            if ((++spins & 0x3Fu) == 0 && (*abort_flag || clock64() - t0 > limit)) {
               *abort_flag = 1;
               raise_status(p.hdr, FASTKV_ERR_DEVICE_TIMEOUT, SITE_FUSED_FLAG);
               break;
@@ -395,7 +407,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         }
       }
       group_sync<2>();
-      if (*abort_flag) break;
+      if (*abort_flag) ok = false;                       // every warp still reaches every barrier below
       // the softmax normaliser of the phase, merged in a fixed order (the same in every CTA)
       merge_buf[bt] = merge_partials(p.partial + static_cast<size_t>(w.stat) * ncta * NPAD, NPAD, bt % NPAD, bt / NPAD,
                                      kParts, w.nact);
@@ -412,9 +424,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       for (int i = 0; i < w.n; ++i, ++it) {
         if ((it & 1) != set) continue;                   // the other set's tile
         const int a = it % kAcc;
-        ok = mbar_wait_bounded(&bars->acc2_full[a], (it / kAcc) & 1, abort_flag, p.hdr, SITE_FUSED_ACC_FULL);
+        if (ok) ok = mbar_wait_bounded(&bars->acc2_full[a], (it / kAcc) & 1, abort_flag, p.hdr, SITE_FUSED_ACC_FULL, limit);
         ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
+        if (!ok) continue;
         tc_fence_after_sync();
         const int key = (w.t0 + i) * kTileKeys + key_in_tile;
         const bool tile_unmasked = (w.t0 + i + 1) * kTileKeys <= win_start;
@@ -540,12 +552,14 @@ template <int D, int NPAD>
 static cudaError_t launch_fused_t(const CUtensorMap& tk, const CUtensorMap& tq, const FusedParams& p, int grid,
                                   cudaStream_t stream) {
   using Cfg = FusedCfg<D, NPAD>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(score_fused_kernel<D, NPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         Cfg::kSmemBytes);
+  static PerDeviceOnce configured;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (!configured.done(dev)) {
+    e = cudaFuncSetAttribute(score_fused_kernel<D, NPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured.set(dev);
   }
   void* args[] = {const_cast<CUtensorMap*>(&tk), const_cast<CUtensorMap*>(&tq), const_cast<FusedParams*>(&p)};
   return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(score_fused_kernel<D, NPAD>), dim3(grid),
@@ -564,12 +578,10 @@ cudaError_t launch_score_fused(int head_dim, int npad, const CUtensorMap& tk, co
 cudaError_t launch_pool_rows(const PoolRowsParams& p, int max_len, int batch, cudaStream_t stream) {
   const int rows = p.n_kv_heads * (p.per_head ? p.group : 1);
   const size_t smem = sizeof(float) * static_cast<size_t>(rows) * (kPoolKeys + 2 * (p.pool_kernel >> 1));
-  static size_t configured = 48 * 1024;
-  if (smem > configured) {
+  if (smem > 48 * 1024) {          // rare (many heads, wide pooling window): opt in on every such launch
     cudaError_t e = cudaFuncSetAttribute(pool_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(smem));
     if (e != cudaSuccess) return e;
-    configured = smem;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((max_len + kPoolKeys - 1) / kPoolKeys, batch);

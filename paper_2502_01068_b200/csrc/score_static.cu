@@ -12,7 +12,7 @@
 
 namespace {
 
-// 16 MiB: enough for the Llama-3.1-8B head shape (8 KV heads, G*w = 32) up to 16 000 tokens.
+// 16 MiB: enough for the Llama-3.1-8B head shape (8 KV heads, G*w = 32) up to about 500 000 tokens.
 // Every GPU on which this library is loaded holds the array until the process exits.
 constexpr size_t kStaticScratchBytes = size_t(16) << 20;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
@@ -61,6 +61,21 @@ int fastkv_score_static(const fastkv_shape* shape, const void* q, const void* k,
   }
   // fastkv_score clears the part of the scratch that must start at zero (status word, counters).
   return fastkv_score(shape, q, k, scores_kv, scores_tsp, scratch, kStaticScratchBytes, stream);
+}
+
+int fastkv_score_static_status(void* stream, int32_t* status, int32_t* site) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+    return fastkv::report_error(FASTKV_ERR_CUDA, "fastkv_score_static_status: no usable current device");
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    scratch = g_scratch_ptr[dev];
+  }
+  if (scratch == nullptr)
+    return fastkv::report_error(FASTKV_ERR_INVALID_ARG,
+                                "fastkv_score_static_status: fastkv_score_static has not run on this device");
+  return fastkv_device_status(scratch, stream, status, site);   // the status word heads the array
 }
 
 }  // extern "C"

@@ -268,7 +268,8 @@ __global__ void __launch_bounds__(THREADS, 1) select_topk_kernel(const SelectPar
       }
     }
   }
-  if (rank == 0 && tid < w) out[k_sel + tid] = n_cand + tid;   // the window, always kept
+  if (rank == 0)
+    for (int i = tid; i < w; i += THREADS) out[k_sel + i] = n_cand + i;   // the window, always kept
   cluster.sync();   // no CTA may exit while others still read its shared memory
 }
 
@@ -277,12 +278,15 @@ namespace {
 template <int CLUSTER, int ITEMS, int THREADS>
 cudaError_t launch_select_t(const SelectParams& p, int batch, cudaStream_t stream) {
   if (CLUSTER > 8) {
-    static bool configured = false;
-    if (!configured) {
-      cudaError_t e = cudaFuncSetAttribute(select_topk_kernel<CLUSTER, ITEMS, THREADS>,
-                                           cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    static PerDeviceOnce configured;      // launch attributes are per device
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (!configured.done(dev)) {
+      e = cudaFuncSetAttribute(select_topk_kernel<CLUSTER, ITEMS, THREADS>,
+                               cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
       if (e != cudaSuccess) return e;
-      configured = true;
+      configured.set(dev);
     }
   }
   cudaLaunchConfig_t cfg = {};

@@ -196,6 +196,19 @@ def make_layer(wl: Workload, layer: int = 0, *, with_v: bool = True, with_hidden
                        cu_seqlens=cu, planted=planted)
 
 
+def full_q(wl: Workload, x: LayerInputs, layer: int = 0) -> np.ndarray:
+    """The packed query tensor [total, Hq, d] of a layer: the rows the method reads (the last w of every
+    sequence) are x.q_win, every other row is an independent N(0,1) draw that must not matter."""
+    total = int(x.cu_seqlens[-1])
+    q = _normal_bf16((wl.cfg, layer, _T_Q, 1), (total, wl.n_q_heads, wl.head_dim))
+    w = wl.window
+    for b in range(len(x.cu_seqlens) - 1):
+        hi = int(x.cu_seqlens[b + 1])
+        if hi - int(x.cu_seqlens[b]) >= w:
+            q[hi - w:hi] = x.q_win[b * w:(b + 1) * w]
+    return q
+
+
 def _llama8b(name: str, cfg: int, seq_lens, k_kv, k_tsp, **kw) -> Workload:
     return Workload(name=name, cfg=cfg, n_q_heads=32, n_kv_heads=8, head_dim=128, hidden_dim=4096,
                     window=8, pool_kernel=7, pool_mode=POOL_AVG, seq_lens=list(seq_lens),

@@ -24,3 +24,18 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture
+def debug_hooks():
+    """Sets the library's process-wide test hooks for one test and puts the defaults back afterwards."""
+    from paper_2502_01068_b200 import binding as B
+    keys = ("score_path", "fused_heads", "fused_lead", "wait_limit_cycles", "extra_publications")
+
+    def set_hook(key, value):
+        assert key in keys
+        B.fastkv_debug_set(key, value)
+
+    yield set_hook
+    for key in keys:
+        B.fastkv_debug_set(key, 0)

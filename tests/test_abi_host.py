@@ -49,8 +49,16 @@ def status_of(fn, *a):
 
 def test_workspace_bytes_and_shape_validation():
     n = B.fastkv_workspace_bytes(good_shape())
-    assert n % 256 == 0 and n > 8 * 32 * 4096 * 4
-    assert B.fastkv_workspace_bytes(good_shape(total_len=131072)) > 8 * 32 * 131072 * 4
+    assert n % 256 == 0 and n > 8 * 4096 * 4
+    # the persistent kernels keep one fp32 row per KV head plus statistics, not the fp32 logits
+    assert 8 * 131072 * 4 < B.fastkv_workspace_bytes(good_shape(total_len=131072)) < 6 * 2 ** 20
+    B.fastkv_debug_set("score_path", 1)                 # the buffered path needs room for the logits
+    try:
+        assert B.fastkv_workspace_bytes(good_shape(total_len=131072)) > 8 * 32 * 131072 * 4
+    finally:
+        B.fastkv_debug_set("score_path", 0)
+    assert status_of(B.fastkv_debug_set, "no_such_key", 1) == B.ERR_INVALID_ARG
+    assert status_of(B.fastkv_debug_set, "score_path", 9) == B.ERR_INVALID_ARG
     assert status_of(B.fastkv_workspace_bytes, good_shape(head_dim=96)) == B.ERR_UNSUPPORTED
     assert status_of(B.fastkv_workspace_bytes, good_shape(window=32)) == B.ERR_UNSUPPORTED      # G*w = 128
     assert status_of(B.fastkv_workspace_bytes, good_shape(n_q_heads=30)) == B.ERR_INVALID_ARG

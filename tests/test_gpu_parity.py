@@ -86,20 +86,24 @@ def test_llama8b_8k():
     assert st["score_err"] < 2e-3
 
 
-def test_buffered_two_pass_path_still_matches(monkeypatch):
-    """Sequences too long for the tensor-memory-resident scoring kernel use the two-pass kernel with
-    buffered logits; FASTKV_SCORE_PATH=buffered selects it for any shape."""
-    monkeypatch.setenv("FASTKV_SCORE_PATH", "buffered")
+@pytest.mark.parametrize("path", [1, 2, 3])
+def test_every_scoring_kernel_matches(debug_hooks, path):
+    """The library picks one of three scoring kernels by shape: (3) logits parked in tensor memory,
+    (2) K read a second time from L2, (1) fp32 logits buffered in the workspace.  Each of them, forced
+    through the score_path hook, must match the oracle on the same layers."""
+    debug_hooks("score_path", path)
     for wl in (W.tiny(), small("buf", 600, [3000, 130, 1000], [300, 64, 200], [500, 20, 100])):
         x = W.make_layer(wl)
         for order in (B.GROUP_THEN_POOL, B.POOL_THEN_GROUP):
             g = gpu_layer(wl, x, pool_mode=B.POOL_MAX, agg_order=order)
             o = oracle_layer(wl, x, pool_mode=B.POOL_MAX, agg_order=order)
-            check_layer(wl, x, g, o, what="buffered")
+            check_layer(wl, x, g, o, what="path %d" % path)
 
 
-def test_sequence_longer_than_tensor_memory_capacity():
-    """L = 160 000 > 148 SMs x 8 tiles x 128 keys: falls back to the buffered path by itself."""
+def test_sequence_longer_than_half_the_tensor_memory_ring():
+    """L = 160 000: a CTA would own 9 tiles per phase, more than half of the 16 parked slots, so the
+    library picks the kernel that re-reads K from L2 by itself; the parked kernel, forced, still works
+    (9 <= 16) and gives the same result up to rounding."""
     wl = small("long", 601, [160000], [4000], [8000], Hq=4, Hkv=1, d=64, hidden=64)
     x = W.make_layer(wl)
     g = gpu_layer(wl, x)
@@ -107,7 +111,23 @@ def test_sequence_longer_than_tensor_memory_capacity():
     check_layer(wl, x, g, o, what="160k")
 
 
-def test_group_sizes_and_wide_windows_on_the_fused_path():
+def test_parked_kernel_at_the_edge_of_its_ring(debug_hooks):
+    debug_hooks("score_path", 3)
+    wl = small("long", 601, [160000], [4000], [8000], Hq=4, Hkv=1, d=64, hidden=64)
+    x = W.make_layer(wl)
+    g = gpu_layer(wl, x)
+    o = oracle_layer(wl, x)
+    check_layer(wl, x, g, o, what="160k parked")
+    # beyond 148 CTAs x 16 slots x 128 keys the parked kernel cannot run: refused on the host
+    shape = B.make_shape(total_len=310000, n_q_heads=4, n_kv_heads=1, head_dim=64)
+    with pytest.raises(B.FastKVError) as e:
+        B.fastkv_workspace_bytes(shape)
+    assert e.value.status == B.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("path", [2, 3])
+def test_group_sizes_and_wide_windows_on_the_persistent_kernels(debug_hooks, path):
+    debug_hooks("score_path", path)
     for Hq, Hkv, w in [(8, 8, 8), (16, 8, 8), (16, 2, 8), (8, 2, 16), (4, 1, 16), (12, 4, 8)]:
         wl = small("grp", 700 + Hq + Hkv + w, [2000], [300], [400], Hq=Hq, Hkv=Hkv, w=w)
         x = W.make_layer(wl)
@@ -117,13 +137,15 @@ def test_group_sizes_and_wide_windows_on_the_fused_path():
             check_layer(wl, x, g, o, what="G=%d w=%d order=%d" % (Hq // Hkv, w, order))
 
 
+@pytest.mark.parametrize("path", [2, 3])
 @pytest.mark.parametrize("scale", [0.5, 2.0])
-def test_wide_logit_range_exercises_reference_rescaling(scale):
+def test_wide_logit_range_exercises_reference_rescaling(debug_hooks, scale, path):
     """With a large softmax scale the logits span far more than the slack the kernel allows between a
     lane's reference and its running maximum, so stored exponentials get rescaled mid-phase.  Scores
     only (most of them underflow to zero on both sides, which makes the selection a tie lottery)."""
     import oracle
     from tests.parity import SCORE_RTOL, dev
+    debug_hooks("score_path", path)
     for L, Hq, Hkv, d, w in [(5000, 8, 2, 128, 8), (1500, 4, 1, 64, 8), (20000, 8, 2, 128, 16)]:
         wl = small("wide", 800 + L, [L], [w], [w], Hq=Hq, Hkv=Hkv, d=d, w=w)
         x = W.make_layer(wl, with_v=False, with_hidden=False)
@@ -140,17 +162,18 @@ def test_wide_logit_range_exercises_reference_rescaling(scale):
         assert np.all(np.abs(s_tsp.cpu().numpy() - ref_tsp) <= SCORE_RTOL * np.abs(ref_tsp) + 1e-12)
 
 
-@pytest.mark.parametrize("heads,lead", [("1", "2"), ("2", "1000"), ("3", "2"), ("8", "3")])
-def test_phase_shapes_of_the_scoring_kernel(monkeypatch, heads, lead):
-    """The persistent scoring kernel cuts its work into phases of `heads` KV heads and lets pass 1 run
-    `lead` phases ahead; the result must not depend on either (tuning knobs forced through the environment)."""
-    monkeypatch.setenv("FASTKV_FUSED_HEADS", heads)
-    monkeypatch.setenv("FASTKV_FUSED_LEAD", lead)
+@pytest.mark.parametrize("heads,lead", [(1, 2), (2, 1000), (3, 2), (8, 3)])
+def test_phase_shapes_of_the_rereading_kernel(debug_hooks, heads, lead):
+    """The kernel that reads K twice cuts its work into phases of `heads` KV heads and lets pass 1 run
+    `lead` phases ahead; the result must not depend on either (tuning hooks of the library)."""
+    debug_hooks("score_path", 2)
+    debug_hooks("fused_heads", heads)
+    debug_hooks("fused_lead", lead)
     wl = small("phases", 900, [20000, 3000], [500, 100], [2000, 300], Hq=32, Hkv=8)
     x = W.make_layer(wl, with_hidden=False)
     g = gpu_layer(wl, x)
     o = oracle_layer(wl, x, do_compact=False)
-    check_layer(wl, x, g, o, what="heads=%s lead=%s" % (heads, lead))
+    check_layer(wl, x, g, o, what="heads=%d lead=%d" % (heads, lead))
 
 
 def test_sequence_shorter_than_the_window_is_reported_not_scored():
@@ -174,3 +197,29 @@ def test_sequence_shorter_than_the_window_is_reported_not_scored():
         lo, hi = int(x.cu_seqlens[b]), int(x.cu_seqlens[b + 1])
         ref, _, _ = oracle.scores(x.q_win[b * 8:(b + 1) * 8], hi - lo - 8, x.k[lo:hi], 8, 7)
         assert np.all(np.abs(got[:, lo:hi] - ref) <= 2e-3 * np.abs(ref) + 1e-12)
+
+
+@pytest.mark.parametrize("path", [0, 1, 2, 3])
+def test_full_query_tensor_layout(debug_hooks, path):
+    """q_layout = FASTKV_Q_FULL: the caller hands over the whole packed query tensor [total, Hq, d] and the
+    library reads rows cu_seqlens[b+1]-w .. cu_seqlens[b+1]-1 itself (Eq. 1's Att[h, N_I-n, .] rows).  Every
+    other query row is random and must not matter: same oracle result as with the window-only layout."""
+    debug_hooks("score_path", path)
+    cases = [small("qfull1", 1100, [3000], [400], [600]),
+             small("qfull2", 1101, [700, 8, 129, 2048, 300], [64, 8, 100, 256, 77], [140, 8, 25, 409, 60]),
+             small("qfull3", 1102, [513], [100], [100], Hq=4, Hkv=1, d=64, w=5)]
+    for wl in cases:
+        x = W.make_layer(wl)
+        o = oracle_layer(wl, x)
+        g = gpu_layer(wl, x, q_layout=B.Q_FULL)
+        check_layer(wl, x, g, o, what="%s Q_FULL path %d" % (wl.name, path))
+        gw = gpu_layer(wl, x, q_layout=B.Q_WINDOW)
+        np.testing.assert_array_equal(g["S_kv"], gw["S_kv"])          # same rows read, same arithmetic
+
+
+def test_full_query_tensor_layout_at_8k():
+    wl = W.llama8b_8k()
+    x = W.make_layer(wl)
+    g = gpu_layer(wl, x, q_layout=B.Q_FULL)
+    o = oracle_layer(wl, x)
+    check_layer(wl, x, g, o, what="8k Q_FULL")
