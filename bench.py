@@ -1,24 +1,27 @@
 #!/usr/bin/env python
 """Benchmark of the FastKV score -> select -> compact layer step on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference] [--tp]
 
 One "step" is one pass of the whole hot path (fastkv_score, fastkv_select = select_kv + select_tsp in
 one launch, fastkv_compact) over one layer of synthetic, seeded input.  The default workload is the
 Llama-3.1-8B-shaped layer at L = 131072 with Token-Selective Propagation (KV retention 10 %, TSP
-rate 20 %).  With N > 1 (torchrun, one rank per GPU) every rank runs its own layer of the same
-shape -- the path partitions over independent layers / requests, so there is no collective on the
-data path -- and the reported value is all ranks' tokens over the slowest rank's time.
+rate 20 %).  With N > 1 every rank (one per GPU; started here when the launcher has not started
+them) runs its own layer of the same shape -- the path partitions over independent layers /
+requests, so there is no collective on the data path -- and the reported value is all ranks' tokens
+over the slowest rank's time.  `--tp` adds the tensor-parallel form of the same layer (KV heads
+sharded over the ranks, one all-reduce of the layer-level score).
 
 Prints one JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle instead.
 """
 from __future__ import annotations
 
 import argparse
-import dataclasses
 import json
 import os
+import socket
 import statistics
+import subprocess
 import sys
 import threading
 import time
@@ -34,17 +37,28 @@ from paper_2502_01068_b200 import workloads as W  # noqa: E402
 METRIC = "context tokens/sec for score+select+compact, per layer"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
+L2_BYTES = 126 * 2 ** 20
+KERNELS = {0: "score", 1: "pool", 2: "select", 3: "compact"}
+KERNEL_SYMBOLS = {"score": "score_parked_kernel / score_fused_kernel", "pool": "pool_rows_kernel",
+                  "select": "select_topk_kernel", "compact": "compact_rows_kernel"}
 
 
 def pick_workload(name: str) -> W.Workload:
     table = {
-        "llama8b_128k_tsp_layer": W.llama8b_128k(),
-        "llama8b_8k": W.llama8b_8k(),
-        "llama8b_32k_tsp_layer": W.llama8b_32k_sweep(),
-        "llama8b_ragged": W.llama8b_ragged(),
-        "tiny": W.tiny(),
+        "llama8b_128k_tsp_layer": W.llama8b_128k,
+        "llama8b_8k": W.llama8b_8k,
+        "llama8b_32k_tsp_layer": W.llama8b_32k_sweep,
+        "llama8b_ragged": W.llama8b_ragged,
+        "tiny": W.tiny,
     }
-    return table[name]
+    return table[name]()
+
+
+def config_of(name: str, wl: W.Workload) -> dict:
+    """What both arms print as `config`."""
+    return {"workload": name, "seq_lens": wl.seq_lens, "k_kv": wl.k_kv, "k_tsp": wl.k_tsp,
+            "n_q_heads": wl.n_q_heads, "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim,
+            "hidden_dim": wl.hidden_dim, "window": wl.window, "pool_kernel": wl.pool_kernel}
 
 
 def algorithmic_bytes(wl: W.Workload) -> dict:
@@ -56,12 +70,15 @@ def algorithmic_bytes(wl: W.Workload) -> dict:
     kt = sum(wl.k_tsp) if wl.k_tsp else 0
     k_read = total * Hkv * d * 2
     q_read = wl.batch * wl.window * wl.n_q_heads * d * 2
+    unpooled = 4 * Hkv * total
     scores = 4 * (Hkv * total + (total if kt else 0))
     idx = 4 * (Hkv * kkv + kt)
     kv_rows = 2 * Hkv * kkv * d * 2
     hid_rows = kt * (hid * 2 + 4)
     return {
-        "score": k_read + q_read + scores,
+        "score": k_read + q_read + scores,                 # the fastkv_score call: both of its kernels
+        "score_kernel": k_read + q_read + unpooled,        # K streamed once, one un-pooled fp32 row per KV head written
+        "pool_kernel": unpooled + scores,
         "select": scores + idx,
         "compact": idx + 2 * kv_rows + 2 * hid_rows,
         "step_rw": k_read + q_read + 2 * scores + 2 * idx + 2 * kv_rows + 2 * hid_rows,
@@ -83,14 +100,16 @@ def profiled_traffic(kernel: str, workload: str):
     tag = {"llama8b_128k_tsp_layer": "llama8b_128k"}.get(workload)
     if tag is None:
         return None
-    path = os.path.join(ROOT, "profiles", "%s_%s.txt" % (kernel, tag))
-    try:
-        with open(path) as f:
-            for line in f:
-                if line.startswith("dram_bytes_per_launch:"):
-                    return int(line.split(":")[1])
-    except OSError:
-        pass
+    for name in {"score": ("score_parked_kernel",), "compact": ("compact_rows_kernel",),
+                 "select": ("select_topk_kernel",), "pool": ("pool_rows_kernel",)}.get(kernel, ()):
+        path = os.path.join(ROOT, "profiles", "%s_%s.txt" % (name, tag))
+        try:
+            with open(path) as f:
+                for line in f:
+                    if line.startswith("dram_bytes_per_launch:"):
+                        return int(line.split(":")[1])
+        except OSError:
+            pass
     return None
 
 
@@ -162,22 +181,96 @@ def whole_job_throughput(tokens_per_rank: int, world: int, ms_per_step: float) -
     return world * tokens_per_rank / (ms_per_step * 1e-3)
 
 
-def oracle_baseline(wl: W.Workload, x: W.LayerInputs, budget_s: float = 15.0, max_reps: int = 16) -> dict:
-    """Times the fp64 oracle, as it stands, on this machine's host cores on the same layer."""
+def spawn_command(n: int, argv, port: int):
+    """The launcher line that starts `n` ranks of this script on one node (what the scaling run uses)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(n: int, argv) -> int:
+    """`--gpus N` without a launcher: start the N ranks here and hand their output through."""
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "WARN")
+    return subprocess.call(spawn_command(n, argv, free_port()), env=env)
+
+
+def oracle_layer_timed(wl: W.Workload, x: W.LayerInputs) -> dict:
+    """One whole layer through the oracle's routines in the order of Algorithm 1, each step timed."""
     import oracle
-    from oracle.layer import layer_step
+    w, t = wl.window, {"scores": 0.0, "select": 0.0, "compact": 0.0}
+    for b in range(wl.batch):
+        lo, hi = int(x.cu_seqlens[b]), int(x.cu_seqlens[b + 1])
+        t0 = time.perf_counter()
+        s_kv, s_tsp, _ = oracle.scores(x.q_win[b * w:(b + 1) * w], hi - lo - w, x.k[lo:hi], w, wl.pool_kernel, wl.pool_mode)
+        t1 = time.perf_counter()
+        idx_kv = [oracle.select(s_kv[g], int(wl.k_kv[b]), w)[0] for g in range(wl.n_kv_heads)]
+        idx_tsp = oracle.select(s_tsp, int(wl.k_tsp[b]), w)[0] if wl.k_tsp else None
+        t2 = time.perf_counter()
+        for g in range(wl.n_kv_heads):
+            oracle.gather_rows(x.k[:, g, :], lo + idx_kv[g])
+            if x.v is not None:
+                oracle.gather_rows(x.v[:, g, :], lo + idx_kv[g])
+        if idx_tsp is not None and x.hidden is not None:
+            oracle.gather_rows(x.hidden, lo + idx_tsp)
+            oracle.gather_rows(x.pos, lo + idx_tsp)
+        t3 = time.perf_counter()
+        t["scores"] += t1 - t0
+        t["select"] += t2 - t1
+        t["compact"] += t3 - t2
+    t["layer"] = t["scores"] + t["select"] + t["compact"]
+    return t
+
+
+ONE_THREAD_CHILD = r"""
+import json, sys, time
+sys.path.insert(0, %r)
+import bench
+from paper_2502_01068_b200 import workloads as W
+wl = bench.pick_workload(%r)
+x = W.make_layer(wl)
+import oracle
+oracle.build()
+t = bench.oracle_layer_timed(wl, x)
+print(json.dumps({"threads": oracle.num_threads(), "seconds": t}))
+"""
+
+
+def oracle_baseline(name: str, wl: W.Workload, x: W.LayerInputs, budget_s: float = 12.0, max_reps: int = 8) -> dict:
+    """Times the fp64 oracle, as it stands, on this machine's host cores on the same layer: with all cores
+    (mean of a few whole layers, per step), and once with a single thread (a child process with
+    OMP_NUM_THREADS=1; skipped when one run would not fit the budget)."""
+    import oracle
     oracle.build()
-    reps, times = 0, []
+    reps, runs = 0, []
     t_all = time.perf_counter()
     while reps < max_reps and (time.perf_counter() - t_all) < budget_s:
-        t0 = time.perf_counter()
-        layer_step(x.q_win, x.k, x.v, x.hidden, x.pos, x.cu_seqlens, wl.window, wl.pool_kernel, wl.k_kv,
-                   wl.k_tsp, pool_mode=wl.pool_mode)
-        times.append(time.perf_counter() - t0)
+        runs.append(oracle_layer_timed(wl, x))
         reps += 1
-    t = statistics.mean(times)
-    return {"value": wl.total_len / t, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": "the whole layer (%d tokens), mean of %d run(s), %.2f s each" % (wl.total_len, reps, t)}
+    t = statistics.mean(r["layer"] for r in runs)
+    steps = {k: statistics.mean(r[k] for r in runs) for k in ("scores", "select", "compact")}
+    out = {"value": wl.total_len / t, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+           "sample": "the whole layer (%d tokens), mean of %d run(s), %.2f s each" % (wl.total_len, reps, t),
+           "seconds_per_step": steps}
+    est_one = t * oracle.num_threads()
+    if est_one <= 45.0:
+        try:
+            env = dict(os.environ, OMP_NUM_THREADS="1")
+            r = subprocess.run([sys.executable, "-c", ONE_THREAD_CHILD % (ROOT, name)], env=env, capture_output=True,
+                               text=True, timeout=240)
+            d = json.loads(r.stdout.strip().splitlines()[-1])
+            out["one_thread"] = {"value": wl.total_len / d["seconds"]["layer"], "unit": UNIT, "cores": d["threads"],
+                                 "seconds_per_step": {k: d["seconds"][k] for k in ("scores", "select", "compact")}}
+        except Exception as e:   # the all-core figure stands on its own
+            out["one_thread"] = {"skipped": "%s" % (e,)}
+    else:
+        out["one_thread"] = {"skipped": "one single-threaded layer would take about %.0f s" % est_one}
+    return out
 
 
 def run_reference(args) -> None:
@@ -190,20 +283,22 @@ def run_reference(args) -> None:
     oracle.build()
     wl = pick_workload(args.workload)
     x = W.make_layer(wl)
+
+    def one():
+        layer_step(x.q_win, x.k, x.v, x.hidden, x.pos, x.cu_seqlens, wl.window, wl.pool_kernel, wl.k_kv, wl.k_tsp,
+                   pool_mode=wl.pool_mode)
+
     # each step is the whole layer; steps are capped so that the run ends within a few minutes
     t0 = time.perf_counter()
-    layer_step(x.q_win, x.k, x.v, x.hidden, x.pos, x.cu_seqlens, wl.window, wl.pool_kernel, wl.k_kv, wl.k_tsp,
-               pool_mode=wl.pool_mode)
-    one = time.perf_counter() - t0
-    warm = max(0, min(args.warmup, int(20.0 / max(one, 1e-3)) - 1))
-    steps = max(1, min(args.steps, int(90.0 / max(one, 1e-3))))
+    one()
+    first = time.perf_counter() - t0
+    warm = max(0, min(args.warmup, int(20.0 / max(first, 1e-3)) - 1))
+    steps = max(1, min(args.steps, int(90.0 / max(first, 1e-3))))
     for _ in range(warm):
-        layer_step(x.q_win, x.k, x.v, x.hidden, x.pos, x.cu_seqlens, wl.window, wl.pool_kernel, wl.k_kv,
-                   wl.k_tsp, pool_mode=wl.pool_mode)
+        one()
     t0 = time.perf_counter()
     for _ in range(steps):
-        layer_step(x.q_win, x.k, x.v, x.hidden, x.pos, x.cu_seqlens, wl.window, wl.pool_kernel, wl.k_kv,
-                   wl.k_tsp, pool_mode=wl.pool_mode)
+        one()
     dt = (time.perf_counter() - t0) / steps
     value = wl.total_len / dt
     sample = "the whole layer per step; %d timed step(s) of %.2f s (requested %d)" % (steps, dt, args.steps)
@@ -211,7 +306,7 @@ def run_reference(args) -> None:
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "seq_lens": wl.seq_lens if wl.batch <= 8 else "ragged"},
+        "config": config_of(args.workload, wl),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -226,13 +321,19 @@ def main() -> None:
     ap.add_argument("--workload", default="llama8b_128k_tsp_layer")
     ap.add_argument("--impl", default="fastkv", choices=["fastkv", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--min-region-s", type=float, default=0.5,
+                    help="the K-step timed region is repeated until this much device time has been measured")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tp", action="store_true",
+                    help="with N > 1: also time the tensor-parallel form (KV heads sharded, one all-reduce of S_tsp)")
     ap.add_argument("--with-decode", action="store_true",
                     help="also time the decode-time attention over the compact cache the step produced")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
         return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))      # one rank per GPU; rank 0 prints the line
 
     import torch
     from paper_2502_01068_b200 import binding as B
@@ -277,21 +378,15 @@ def main() -> None:
     hid_out = torch.empty((b_tsp.total, wl.hidden_dim), dtype=torch.int16, device="cuda")
     pos_out = torch.empty((b_tsp.total,), dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream()
+    input_bytes = x.k.nbytes + x.v.nbytes + x.hidden.nbytes
+    fits_l2 = x.k.nbytes + x.q_win.nbytes <= L2_BYTES       # then "HBM GB/s" needs an L2 flush between steps
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if fits_l2 else None
 
-    def step(events=None):
-        if events is not None:
-            events[0].record(stream)
+    def step():
         B.fastkv_score(shape, q, k, s_kv, s_tsp, ws, stream)
-        if events is not None:
-            events[1].record(stream)
         B.fastkv_select(shape, s_kv, b_kv, idx_kv, s_tsp, b_tsp, idx_tsp, ws, stream)   # select_kv + select_tsp
-        if events is not None:
-            events[2].record(stream)
-            events[3].record(stream)
         B.fastkv_compact(shape, idx_kv, b_kv, idx_tsp, b_tsp, k, v, hid, pos, k_out, v_out, hid_out, pos_out, ws,
                          stream)
-        if events is not None:
-            events[4].record(stream)
 
     def barrier():
         if world > 1:
@@ -305,34 +400,74 @@ def main() -> None:
     if status != 0:
         raise SystemExit("device status %d at site %d after warm-up" % (status, site))
 
-    # ---- timed region: K steps back to back, device-timed from the first launch to the last kernel's end ---------
+    def timed_region() -> float:
+        """Exactly K steps, device-timed from the first launch to the last kernel's end, in ms.  Workloads whose
+        inputs fit in L2 get the L2 overwritten before every step (not timed) and are timed step by step."""
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        torch.cuda.synchronize()
+        if flush is None:
+            t0.record(stream)
+            for _ in range(steps):
+                step()
+            t1.record(stream)
+            torch.cuda.synchronize()
+            ms = t0.elapsed_time(t1)
+        else:
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+            for a, b in ev:
+                flush.zero_()
+                a.record(stream)
+                step()
+                b.record(stream)
+            torch.cuda.synchronize()
+            ms = sum(a.elapsed_time(b) for a, b in ev)
+        barrier()
+        return ms
+
+    # ---- timed region: K steps, repeated until enough device time has been measured; the median repeat is reported -----
     sampler = ClockSampler(local_rank)
-    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = B.fastkv_kernel_launches()
-    barrier()
-    torch.cuda.synchronize()
     sampler.start()
-    t_begin.record(stream)
-    for i in range(steps):
-        step()
-    t_end.record(stream)
-    torch.cuda.synchronize()
-    barrier()
+    region_ms = [timed_region()]
     launches = B.fastkv_kernel_launches() - launches0
-    total_ms = t_begin.elapsed_time(t_end)
-    # ---- the same K steps again with an event between the calls: per-call durations for the roofline objects.
-    # An event record between two kernels keeps the second from starting under the first one's tail (programmatic
-    # dependent launch), so this loop is a few percent slower than the timed one; both are reported.
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
-    for i in range(steps):
-        step(ev[i])
-    torch.cuda.synchronize()
-    clocks = sampler.stop()
-    instrumented_ms = ev[0][0].elapsed_time(ev[-1][4]) / steps
-    call_ms = [statistics.mean(ev[i][c].elapsed_time(ev[i][c + 1]) for i in range(steps)) for c in range(4)]
-    total_ms = max_over_ranks(total_ms, world, "cuda")
+    n_rep = int(min(400, max(1, np.ceil(args.min_region_s * 1e3 / max(region_ms[0], 1e-3)))))
+    n_rep = int(max_over_ranks(n_rep, world, "cuda"))
+    for _ in range(n_rep - 1):
+        region_ms.append(timed_region())
+    region_ms = [max_over_ranks(t, world, "cuda") for t in region_ms]
+    total_ms = statistics.median(region_ms)
     ms_per_step = total_ms / steps
     value = whole_job_throughput(total, world, ms_per_step)
+
+    # ---- L2-warm variant for the workloads that fit in L2 (same K steps back to back, no flush) -------------------------
+    warm_ms = None
+    if flush is not None:
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t0.record(stream)
+        for _ in range(steps):
+            step()
+        t1.record(stream)
+        torch.cuda.synchronize()
+        warm_ms = max_over_ranks(t0.elapsed_time(t1), world, "cuda") / steps
+
+    # ---- the same K steps with a pair of events around every kernel (the library's own hook): per-kernel durations.
+    # An event between two kernels keeps the second from starting under the first one's tail (programmatic dependent
+    # launch), so these add up to a little more than a step of the timed region.
+    B.fastkv_debug_set("time_kernels", 1)
+    for _ in range(steps):
+        if flush is not None:
+            flush.zero_()
+        step()
+    torch.cuda.synchronize()
+    B.fastkv_debug_set("time_kernels", 0)
+    clocks = sampler.stop()
+    kernel_ms = {}
+    for kid, kname in KERNELS.items():
+        _, ms, n = B.fastkv_debug_kernel_time(kid)
+        if n:
+            kernel_ms[kname] = ms / n
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies timed) -------------
     e2e = None
@@ -369,8 +504,40 @@ def main() -> None:
         d2h = sum(t.numel() * t.element_size() for t in (o_idx_kv, o_idx_tsp, o_k, o_v, o_h, o_p))
         e2e = {"value": world * total / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "ms_per_step": e2e_s * 1e3, "steps": args.e2e_steps}
-        if np.array_equal(o_idx_tsp.numpy(), idx_tsp.cpu().numpy()) is False:
-            raise SystemExit("host-buffer path and device path disagree on idx_tsp")
+        same = (np.array_equal(o_idx_tsp.numpy(), idx_tsp.cpu().numpy()) and
+                np.array_equal(o_idx_kv.numpy(), idx_kv.cpu().numpy()) and
+                np.array_equal(o_k.numpy(), k_out.cpu().numpy()) and np.array_equal(o_h.numpy(), hid_out.cpu().numpy()))
+        if not same:
+            raise SystemExit("host-buffer path and device path disagree")
+
+    # ---- optional: tensor-parallel form of the same layer (KV heads sharded, one all-reduce of S_tsp) -------------------
+    tp = None
+    if args.tp and world > 1 and Bn == 1 and wl.n_kv_heads % world == 0:
+        from paper_2502_01068_b200.tp import CudaBackend, HeadShard, shard_heads, tp_layer_step
+        x0 = W.make_layer(wl, layer=0)                     # every rank draws the same layer and keeps its heads
+        shard = HeadShard(rank, world, wl.n_q_heads, wl.n_kv_heads)
+        backend = CudaBackend(shard, total, wl.head_dim, wl.hidden_dim, wl.window, wl.pool_kernel, wl.pool_mode)
+        tq, tk, tv = (shard_heads(tdev(a), r) for a, r in ((x0.q_win, shard.q_range), (x0.k, shard.kv_range),
+                                                            (x0.v, shard.kv_range)))
+        th, tpos = tdev(x0.hidden), tdev(x0.pos)
+        kk, kt = int(wl.k_kv[0]), int(wl.k_tsp[0])
+        for _ in range(3):
+            out = tp_layer_step(backend, shard, tq, tk, tv, th, tpos, kk, kt)
+        barrier()
+        torch.cuda.synchronize()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(steps):
+            out = tp_layer_step(backend, shard, tq, tk, tv, th, tpos, kk, kt)
+        t1.record(stream)
+        torch.cuda.synchronize()
+        tp_ms = max_over_ranks(t0.elapsed_time(t1), world, "cuda") / steps
+        gathered = [torch.zeros_like(out[1]) for _ in range(world)]
+        import torch.distributed as dist
+        dist.all_gather(gathered, out[1])
+        tp = {"ms_per_step": tp_ms, "value": total / (tp_ms * 1e-3), "unit": UNIT, "scaling": "strong",
+              "kv_heads_per_rank": shard.local_kv_heads, "all_reduce_bytes": 4 * total,
+              "same_idx_tsp_on_all_ranks": all(bool(torch.equal(g, out[1])) for g in gathered)}
 
     # ---- optional: decode-time attention of one new token over the compacted cache of this layer ------------------
     decode = None
@@ -378,10 +545,10 @@ def main() -> None:
         qd = torch.randn((Bn, wl.n_q_heads, wl.head_dim), device="cuda").to(torch.bfloat16).view(torch.int16)
         dws = torch.empty(B.fastkv_decode_attn_workspace_bytes(shape), dtype=torch.uint8, device="cuda")
         dout = torch.empty((Bn, wl.n_q_heads, wl.head_dim), dtype=torch.float32, device="cuda")
-        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # the cache alone would fit in L2
+        dflush = flush if flush is not None else torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
         times = []
         for i in range(13):
-            flush.zero_()
+            dflush.zero_()                                # the cache alone would fit in L2
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
             B.fastkv_decode_attn(shape, qd, k_out, v_out, b_kv, dout, None, dws, stream)
@@ -394,41 +561,54 @@ def main() -> None:
         decode = {"ms": dms, "algorithmic_bytes": dbytes, "achieved_gbs": dbytes / (dms * 1e-3) / 1e9,
                   "frac_of_measured": dbytes / (dms * 1e-3) / 1e9 / measured_peaks()["hbm_gbs"],
                   "l2": "flushed between iterations (256 MB write)", "kept_per_head": int(wl.k_kv[0])}
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
     if rank != 0:
         return
     ab = algorithmic_bytes(wl)
     peaks = measured_peaks()
-    compact_gbs = ab["compact"] / (call_ms[3] * 1e-3) / 1e9
+    kbytes = {"score": ab["score_kernel"], "pool": ab["pool_kernel"], "select": ab["select"], "compact": ab["compact"]}
+
+    def roof(kname: str) -> dict:
+        gbs = kbytes[kname] / (kernel_ms[kname] * 1e-3) / 1e9
+        return {"bound": "hbm", "kernel": KERNEL_SYMBOLS[kname], "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "algorithmic_bytes": kbytes[kname],
+                "traffic": profiled_traffic(kname, args.workload), "ms": kernel_ms[kname],
+                "share_of_kernel_time": kernel_ms[kname] / sum(kernel_ms.values())}
+
+    dominant = max(kernel_ms, key=kernel_ms.get)
     step_gbs = ab["step_rw"] / (ms_per_step * 1e-3) / 1e9
+    config = config_of(args.workload, wl)
+    config["l2"] = ("L2 overwritten (256 MB write) before every step, not timed: the inputs (%.0f MB of K) fit in L2"
+                    % (x.k.nbytes / 1e6)) if flush is not None else (
+        "inputs larger than L2 (K %.0f MB, hidden %.0f MB per step)" % (x.k.nbytes / 1e6, x.hidden.nbytes / 1e6))
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, "seq_lens": lens, "k_kv": wl.k_kv, "k_tsp": wl.k_tsp,
-                   "n_q_heads": wl.n_q_heads, "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim,
-                   "hidden_dim": wl.hidden_dim, "window": wl.window, "pool_kernel": wl.pool_kernel,
-                   "l2": "inputs larger than L2 (K %.0f MB, hidden %.0f MB per step)" % (
-                       x.k.nbytes / 1e6, x.hidden.nbytes / 1e6)},
+        "dtype": "bf16", "data": "synthetic", "config": config,
+        "repeats": {"n": len(region_ms), "ms_per_step_median": ms_per_step, "ms_per_step_min": min(region_ms) / steps,
+                    "ms_per_step_max": max(region_ms) / steps,
+                    "ms_times_sm_mhz": ms_per_step * clocks["sm_mhz"] if clocks.get("sm_mhz") else None},
         "clocks": clocks,
         "gpu_launches": int(launches),
         "e2e": e2e,
-        "roofline": {"bound": "hbm", "kernel": "compact_rows_kernel", "achieved": compact_gbs,
-                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": compact_gbs / peaks["hbm_gbs"],
-                     "peak_source": peaks["source"], "algorithmic_bytes": ab["compact"],
-                     "traffic": profiled_traffic("compact_rows_kernel", args.workload),
-                     "ms": call_ms[3]},
+        "roofline": roof(dominant),
+        "roofline_compact": roof("compact") if "compact" in kernel_ms else None,
         "step_roofline": {"bytes_rw": ab["step_rw"], "bytes_rows_once": ab["step_min"], "achieved_gbs": step_gbs,
                           "frac_of_measured": step_gbs / peaks["hbm_gbs"],
                           "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
                           "rows_once_gbs": ab["step_min"] / (ms_per_step * 1e-3) / 1e9},
-        "calls_ms": {"fastkv_score": call_ms[0], "fastkv_select": call_ms[1], "fastkv_compact": call_ms[3],
-                     "step_with_events_between_calls": instrumented_ms},
-        "calls_gbs": {"fastkv_score": ab["score"] / (call_ms[0] * 1e-3) / 1e9},
+        "kernels_ms": kernel_ms,
     }
+    if warm_ms is not None:
+        line["l2_warm"] = {"ms_per_step": warm_ms, "value": whole_job_throughput(total, world, warm_ms)}
+    if tp is not None:
+        line["tensor_parallel"] = tp
     if decode is not None:
         line["decode_attn"] = decode
     if not args.no_cpu_baseline:
-        line["cpu_baseline"] = oracle_baseline(wl, x)
+        line["cpu_baseline"] = oracle_baseline(args.workload, wl, x)
     print(json.dumps(line))
 
 

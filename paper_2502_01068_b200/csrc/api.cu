@@ -133,15 +133,18 @@ Layout make_layout(const fastkv_shape& s) {
   l.f_off_a = off;
   off += round_up(sizeof(float) * static_cast<size_t>(l.f_rows) * l.ld_logits, 256);
   l.f_bytes = off;
-  // Which kernel scores this shape.  The parked kernel is the fastest while a CTA's tiles of two phases
-  // fit in its tensor-memory ring; longer sequences re-read K from L2 with the two-pipeline kernel; the
-  // buffered two-kernel path serves the remaining shapes.
+  // Which kernel scores this shape.  The parked kernel is the fastest for long sequences, as long as a CTA's
+  // tiles of two phases fit in its tensor-memory ring (measured on a B200 with the Llama-3.1-8B head shape:
+  // 64 us against 89 us at 131072 tokens); it pays a few microseconds per phase, so below about six tiles per
+  // CTA and phase (57 us against 51 us at 65536 tokens, 37 against 18 at 8192), and beyond the ring, the
+  // two-pipeline kernel that reads K a second time from L2 is used; the buffered two-kernel path serves the
+  // remaining shapes.
   const int per = parked_tiles_per_cta(s.max_len, kFusedMaxCtas), slots = parked_slots(l.npad);
   switch (g_debug.score_path) {
     case PATH_BUFFERED: l.path = PATH_BUFFERED; break;
     case PATH_REREAD: l.path = l.fused_shape_ok ? PATH_REREAD : PATH_BUFFERED; break;
     case PATH_PARKED: l.path = !l.fused_shape_ok ? PATH_BUFFERED : (per <= slots ? PATH_PARKED : -1); break;
-    default: l.path = !l.fused_shape_ok ? PATH_BUFFERED : (2 * per <= slots ? PATH_PARKED : PATH_REREAD); break;
+    default: l.path = !l.fused_shape_ok ? PATH_BUFFERED : (per >= 6 && 2 * per <= slots ? PATH_PARKED : PATH_REREAD); break;
   }
   l.bytes = l.path == PATH_BUFFERED ? l.b_bytes : l.f_bytes;
   return l;

@@ -136,3 +136,21 @@ def test_head_shard_arithmetic():
     assert list(s.kv_range) == [2, 3] and list(s.q_range) == list(range(8, 16)) and s.group == 4
     with pytest.raises(ValueError):
         HeadShard(0, 3, 32, 8)
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did():
+    """`bench.py --gpus N` without WORLD_SIZE re-executes itself under the torch launcher with N ranks on
+    127.0.0.1.  Checked here on CPU with the oracle arm on the tiny workload: rank 0 prints the one JSON line,
+    the other rank exits 0 without work."""
+    import json
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.spawn_command(2, ["--impl", "reference", "--workload", "tiny", "--steps", "1", "--warmup", "0", "--gpus", "2"],
+                              free_port())
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "127.0.0.1" in cmd and "2" in cmd
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    r = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-3000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2
+    assert lines[0]["config"] == bench.config_of("tiny", bench.pick_workload("tiny"))
