@@ -326,8 +326,8 @@ def main() -> None:
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tp", action="store_true",
                     help="with N > 1: also time the tensor-parallel form (KV heads sharded, one all-reduce of S_tsp)")
-    ap.add_argument("--with-decode", action="store_true",
-                    help="also time the decode-time attention over the compact cache the step produced")
+    ap.add_argument("--no-decode", action="store_true",
+                    help="skip the decode-time attention over the compact cache the step produced")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -541,7 +541,7 @@ def main() -> None:
 
     # ---- optional: decode-time attention of one new token over the compacted cache of this layer ------------------
     decode = None
-    if args.with_decode and len(set(wl.k_kv)) == 1:
+    if not args.no_decode and len(set(wl.k_kv)) == 1:
         qd = torch.randn((Bn, wl.n_q_heads, wl.head_dim), device="cuda").to(torch.bfloat16).view(torch.int16)
         dws = torch.empty(B.fastkv_decode_attn_workspace_bytes(shape), dtype=torch.uint8, device="cuda")
         dout = torch.empty((Bn, wl.n_q_heads, wl.head_dim), dtype=torch.float32, device="cuda")

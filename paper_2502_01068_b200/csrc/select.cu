@@ -2,8 +2,9 @@
 //
 // One thread-block cluster per problem (one score row of one sequence).  The k-th largest
 // candidate score is found exactly by a most-significant-digit-first radix search on the
-// order-preserving integer image of the fp32 scores (4 passes of 8 bits); per-CTA digit
-// histograms are merged through distributed shared memory.  The kept positions are then
+// order-preserving integer image of the fp32 scores (4 passes of 8 bits); every CTA adds its
+// digit histogram into every CTA's copy of the cluster's histogram with remote shared-memory
+// atomics (nothing waits for them), so after the pass's cluster barrier the sum is local.  The kept positions are then
 // written in ascending order by an index-ordered stream compaction: every candidate above
 // the threshold, plus the lowest-index candidates equal to it until the budget is met --
 // which is exactly "rank by (score descending, index ascending), keep the first k".  With
@@ -32,10 +33,9 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 
 struct alignas(16) SelShared {
   int hist[kBins * 32];          // lane-private digit counters: hist[bin * 32 + lane]
-  int block_hist[2][kBins];      // this CTA's histogram, double-buffered by pass parity
-  int total_hist[kBins];         // the cluster's histogram of the current pass
+  int total_hist[2][kBins];      // the cluster's histogram of a pass (every CTA adds into it), double-buffered by pass parity
   int warp_tot[2][kSelWarps];
-  alignas(8) int counts[2];      // this CTA's (#above threshold, #equal to threshold)
+  alignas(8) int counts[16][2];  // per CTA of the cluster: (#above threshold, #equal to threshold), written by that CTA
   int digit, k_rem;
 };
 
@@ -60,6 +60,8 @@ __global__ void __launch_bounds__(THREADS, 1) select_topk_kernel(const SelectPar
   const int row = static_cast<int>(blockIdx.y) - (second ? p.set[0].n_rows : 0), b = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+  for (int i = tid; i < 2 * kBins; i += THREADS) (&sh.total_hist[0][0])[i] = 0;
+  cluster.sync();              // nobody adds into a histogram that is not cleared yet (overlaps the previous kernel's tail)
   pdl_wait();                  // the scores come from the kernel before this one
   pdl_launch_dependents();
   const int row0 = p.cu_seqlens ? p.cu_seqlens[b] : 0;
@@ -136,21 +138,17 @@ __global__ void __launch_bounds__(THREADS, 1) select_topk_kernel(const SelectPar
         }
         if (kPerBin >= 2) sum += __shfl_xor_sync(0xffffffffu, sum, 1);
         if (kPerBin >= 4) sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-        if (part == 0) sh.block_hist[pass & 1][bin] = sum;
+        if (part == 0 && sum != 0) {   // non-empty bins go to every CTA of the cluster
+#pragma unroll
+          for (int r = 0; r < CLUSTER; ++r) atomicAdd(cluster.map_shared_rank(&sh.total_hist[pass & 1][bin], r), sum);
+        }
       }
       cluster.sync();
-      if (tid < kBins) {               // one bin per thread: sum it over the cluster (DSMEM reads)
-        int c = 0;
-#pragma unroll
-        for (int r = 0; r < CLUSTER; ++r) c += cluster.map_shared_rank(&sh.block_hist[pass & 1][0], r)[tid];
-        sh.total_hist[tid] = c;
-      }
-      __syncthreads();
       if (warp == 0) {
         // 8 bins per lane, highest bins first: lane 0 owns bins 255..248
         int cnt[8], tot = 0;
-        const int4 lo = *reinterpret_cast<const int4*>(&sh.total_hist[248 - lane * 8]);
-        const int4 hi = *reinterpret_cast<const int4*>(&sh.total_hist[252 - lane * 8]);
+        const int4 lo = *reinterpret_cast<const int4*>(&sh.total_hist[pass & 1][248 - lane * 8]);
+        const int4 hi = *reinterpret_cast<const int4*>(&sh.total_hist[pass & 1][252 - lane * 8]);
         cnt[0] = hi.w; cnt[1] = hi.z; cnt[2] = hi.y; cnt[3] = hi.x;
         cnt[4] = lo.w; cnt[5] = lo.z; cnt[6] = lo.y; cnt[7] = lo.x;
 #pragma unroll
@@ -174,6 +172,7 @@ __global__ void __launch_bounds__(THREADS, 1) select_topk_kernel(const SelectPar
         }
       }
       __syncthreads();
+      if (tid < kBins) sh.total_hist[pass & 1][tid] = 0;   // for the pass after next; nobody adds into it before the next barrier
       const uint32_t digit = static_cast<uint32_t>(sh.digit);
       prefix |= digit << shift;
       k_rem = sh.k_rem;
@@ -225,7 +224,9 @@ __global__ void __launch_bounds__(THREADS, 1) select_topk_kernel(const SelectPar
     }
     sh.warp_tot[0][lane] = a - a0;
     sh.warp_tot[1][lane] = e - e0;
-    if (lane == 31) { sh.counts[0] = a; sh.counts[1] = e; }
+    // this CTA's totals go to every CTA of the cluster (remote stores; the barrier below makes them visible)
+    const int a_tot = __shfl_sync(0xffffffffu, a, 31), e_tot = __shfl_sync(0xffffffffu, e, 31);
+    if (lane < CLUSTER) *reinterpret_cast<int2*>(cluster.map_shared_rank(&sh.counts[rank][0], lane)) = make_int2(a_tot, e_tot);
   }
   __syncthreads();
   const int gt_excl = sh.warp_tot[0][warp] + gt_incl - n_gt, eq_excl = sh.warp_tot[1][warp] + eq_incl - n_eq;
@@ -233,10 +234,9 @@ __global__ void __launch_bounds__(THREADS, 1) select_topk_kernel(const SelectPar
   // candidates kept by lower-ranked CTAs (they hold lower indices)
   int g_r[CLUSTER], e_r[CLUSTER];
 #pragma unroll
-  for (int r = 0; r < CLUSTER; ++r) {              // all remote reads in flight at once
-    const int2 c = *reinterpret_cast<const int2*>(cluster.map_shared_rank(&sh.counts[0], r));
-    g_r[r] = c.x;
-    e_r[r] = c.y;
+  for (int r = 0; r < CLUSTER; ++r) {
+    g_r[r] = sh.counts[r][0];
+    e_r[r] = sh.counts[r][1];
   }
   int eq_before = 0, kept_before = 0;
 #pragma unroll
@@ -270,7 +270,7 @@ __global__ void __launch_bounds__(THREADS, 1) select_topk_kernel(const SelectPar
   }
   if (rank == 0)
     for (int i = tid; i < w; i += THREADS) out[k_sel + i] = n_cand + i;   // the window, always kept
-  cluster.sync();   // no CTA may exit while others still read its shared memory
+  // nobody touches another CTA's shared memory after the last barrier above: a CTA may end on its own
 }
 
 namespace {
