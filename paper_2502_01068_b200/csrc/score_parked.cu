@@ -20,9 +20,12 @@
 //              parked for this phase are rescaled) only if a logit exceeds it by more than 64
 //              binary orders of magnitude;
 //   publisher  (one warp) writes the CTA's (max, sum) per row of a finished phase to global memory and
-//              bumps the phase's counter, so that publication never waits behind anything else;
-//   pass 2     (four warps, one per tensor-memory lane quarter) waits until every CTA of the phase
-//              has published, merges the statistics in a fixed order (identical in every CTA:
+//              bumps the phase's counter, so that publication never waits behind anything else; between
+//              publications it watches the counter of the oldest phase not yet collected and, once
+//              every CTA has published, brings all CTAs' statistics of that phase into shared memory
+//              with one bulk copy -- while pass 2 is still busy with the phase before;
+//   pass 2     (four warps, one per tensor-memory lane quarter) waits for the collected statistics
+//              of the phase, merges them in a fixed order (identical in every CTA:
 //              deterministic) into the softmax normaliser of every row, forms one weight per
 //              (key lane, query row), f = exp2(ref - M_r) / l_r, and then only needs a multiply-add
 //              per parked value: the score of a key is the sum of e * f over its window rows and
@@ -55,6 +58,7 @@ constexpr int kPass2Threads = 32 * kPass2Warps;
 constexpr int kParkedThreads = 32 * (kCtrlWarps + kPass1Warps + kPass2Warps);   // 15 warps: at most 4 per scheduler
 constexpr int kMaxStages = 8;
 constexpr int kMaxSlots = 16;
+constexpr int kMaxCtas = 148;                  // CTAs whose statistics the collection buffer holds
 // Pass 1 keeps e = exp2(s - ref) with the row's first logit as the reference; the reference only moves
 // when a logit exceeds it by more than this many binary orders of magnitude (e and its row sums stay far
 // inside the fp32 range: e <= 2^64, at most 2^20-odd terms per sum).
@@ -65,13 +69,17 @@ struct ParkedCfg {
   static constexpr int KH = D / 64;
   static constexpr int kStageBytes = KH * kHalfBytes;
   static constexpr int kQBytes = KH * NPAD * 128;
-  static constexpr int kStages = (D == 128) ? (NPAD == 32 ? 5 : 3) : (NPAD == 32 ? 8 : 6);
+  static constexpr int kStages = (D == 128) ? 3 : 6;
+  // with 32 query rows all CTAs' statistics of a phase (37 KB) are collected in shared memory by the
+  // publisher warp; with 64 rows there is no room and pass 2 reads them from global memory itself
+  static constexpr bool kCollect = NPAD == 32;
+  static constexpr int kCollectBytes = kCollect ? kMaxCtas * NPAD * 8 : 0;
   static constexpr int kSlots = 512 / NPAD;                 // tensor memory: 512 columns
   static constexpr int kBarBytes = 1024;
   static constexpr int kRefBytes = NPAD * kTileKeys * 4;    // one reference per (query row, key lane)
   static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 2 * kQBytes + 2 * kRefBytes + kBarBytes +
                                     2 * 4 * NPAD * 8 /*warp_stats*/ + NPAD * 8 /*norm*/ +
-                                    2 * kPass2Threads * 8 /*merge_buf*/ + NPAD * 4 /*row_j*/;
+                                    2 * kPass2Threads * 8 /*merge_buf*/ + NPAD * 4 /*row_j*/ + kCollectBytes;
 };
 
 struct ParkedBarriers {
@@ -82,6 +90,8 @@ struct ParkedBarriers {
   uint64_t ref_free[2];        // pass 2 has finished with the references of a phase
   uint64_t stats_ready[2];     // pass 1 has written its warps' statistics of a phase
   uint64_t stats_free[2];      // ... and the publisher has read them
+  uint64_t coll_full;          // all CTAs' statistics of a phase have landed in shared memory
+  uint64_t coll_free;          // ... and pass 2 has merged them
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -113,6 +123,27 @@ __device__ __forceinline__ void merge_partials_2rows(const float2* part, int npa
   }
   out0 = make_float2(m0, l0);
   out1 = make_float2(m1, l1);
+}
+
+// The same merge from the copy of all CTAs' statistics in shared memory.
+__device__ __forceinline__ void merge_collected_2rows(const float2* part, int npad, int n2, int first, int stride,
+                                                      int count, float2& out0, float2& out1) {
+  float m0 = -INFINITY, l0 = 0.0f, m1 = -INFINITY, l1 = 0.0f;
+  for (int r = first; r < count; r += stride) {
+    const float4 v = *reinterpret_cast<const float4*>(&part[r * npad + n2]);
+    merge_stats(m0, l0, v.x, v.y);
+    merge_stats(m1, l1, v.z, v.w);
+  }
+  out0 = make_float2(m0, l0);
+  out1 = make_float2(m1, l1);
+}
+
+// global -> shared bulk copy (16-byte aligned, size a multiple of 16) that completes on an mbarrier
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(smem_dst)),
+               "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
 }
 
 template <int GG>
@@ -171,6 +202,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
   float2* norm = warp_stats + 2 * 4 * NPAD;                           // [NPAD] (-row max, 1 / row sum)
   float2* merge_buf = norm + NPAD;                                    // [256] partial merges
   int* row_j = reinterpret_cast<int*>(merge_buf + 2 * kPass2Threads); // [NPAD] window row j = n / G of query row n
+  float2* collected = reinterpret_cast<float2*>(row_j + NPAD);        // [CTAs][NPAD] (16-byte aligned)
   constexpr int CPW = NPAD / 2;                                       // accumulator columns per pass-1 warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -178,7 +210,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
   const long long limit = p.wait_limit;
 
   // A phase that does not fit in the slot ring could never complete: refuse before any barrier exists.
-  if ((((p.max_len + kTileKeys - 1) / kTileKeys) + ncta - 1) / ncta > kSlots) {
+  if ((((p.max_len + kTileKeys - 1) / kTileKeys) + ncta - 1) / ncta > kSlots || ncta > kMaxCtas) {
     if (cta == 0 && threadIdx.x == 0) raise_status(p.hdr, FASTKV_ERR_UNSUPPORTED, SITE_PARKED_RING);
     return;
   }
@@ -196,6 +228,8 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
       mbar_init(&bars->stats_ready[i], kPass1Warps);
       mbar_init(&bars->stats_free[i], 1);
     }
+    mbar_init(&bars->coll_full, 1);
+    mbar_init(&bars->coll_free, 1);
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -296,31 +330,84 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
       }
     }
   } else if (warp == 2) {
-    // ---------------- publisher: this CTA's row statistics of each finished phase go to global memory ----------------
-    int u = 0;
+    // ---------------- publisher: this CTA's row statistics of each finished phase go to global memory; ----------------
+    // ---------------- collector: all CTAs' statistics of a complete phase come back into shared memory ----------------
+    // Two walks over the phase list, `pw` for publication and `cw` for collection; whichever has something to
+    // do goes first, so a publication never waits behind a collection and the other way round.
+    int pu = 0, cu = 0;                                  // phases with tiles here: published / collected
     bool ok = true;
-    PhaseIter pit = {0, 0};
-    PhaseWork w;
-    while (next_phase(p, pit, cta, ncta, w)) {
-      if (w.n == 0) continue;
-      const int buf = u & 1;
-      if (ok) ok = mbar_wait_bounded(&bars->stats_ready[buf], (u >> 1) & 1, abort_flag, p.hdr, SITE_PARKED_STATS, limit);
-      ok = __all_sync(0xffffffffu, ok);
-      const float2* ws = warp_stats + buf * 4 * NPAD;
+    PhaseIter pit = {0, 0}, cit = {0, 0};
+    PhaseWork pw, cw;
+    bool have_p = next_phase(p, pit, cta, ncta, pw), have_c = Cfg::kCollect && next_phase(p, cit, cta, ncta, cw);
+    while (have_p && pw.n == 0) have_p = next_phase(p, pit, cta, ncta, pw);
+    while (have_c && cw.n == 0) have_c = next_phase(p, cit, cta, ncta, cw);
+    long long t0 = clock64();
+    unsigned spins = 0;
+    while (have_p || have_c) {
+      bool progress = false;
+      if (have_p) {
+        const int buf = pu & 1;
+        int ready = 1;
+        if (ok && lane == 0) ready = mbar_try_wait(&bars->stats_ready[buf], (pu >> 1) & 1) ? 1 : 0;
+        ready = __shfl_sync(0xffffffffu, ready, 0);
+        if (ready) {                                     // (an aborted CTA publishes without waiting: nobody hangs on it)
+          __syncwarp();
+          const float2* ws = warp_stats + buf * 4 * NPAD;
 #pragma unroll
-      for (int n = lane; n < NPAD; n += 32) {            // lane quarters -> CTA
-        float mm = -INFINITY, ll = 0.0f;
+          for (int n = lane; n < NPAD; n += 32) {        // lane quarters -> CTA
+            float mm = -INFINITY, ll = 0.0f;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) merge_stats(mm, ll, ws[q * NPAD + n].x, ws[q * NPAD + n].y);
-        p.partial[(static_cast<size_t>(w.stat) * ncta + cta) * NPAD + n] = make_float2(mm, ll);
+            for (int q = 0; q < 4; ++q) merge_stats(mm, ll, ws[q * NPAD + n].x, ws[q * NPAD + n].y);
+            p.partial[(static_cast<size_t>(pw.stat) * ncta + cta) * NPAD + n] = make_float2(mm, ll);
+          }
+          __syncwarp();
+          if (lane == 0) {
+            red_release_add(p.counters + pw.stat, 1);    // release: cumulative over the warp's stores
+            mbar_arrive(&bars->stats_free[buf]);
+          }
+          ++pu;
+          do have_p = next_phase(p, pit, cta, ncta, pw); while (have_p && pw.n == 0);
+          progress = true;
+        }
       }
-      __syncwarp();
-      if (lane == 0) {
-        red_release_add(p.counters + w.stat, 1);         // release: cumulative over the warp's stores
-        mbar_arrive(&bars->stats_free[buf]);
+      if (have_c && !ok) have_c = false;                 // aborted: nothing more is collected
+      if (have_c && cu < pu) {
+        int ready = 0;
+        if (lane == 0)                                   // the buffer is free again and every CTA has published?
+          ready = (mbar_try_wait(&bars->coll_free, (cu & 1) ^ 1) &&
+                   ld_acquire(p.counters + cw.stat) >= cw.nact + p.extra_publications) ? 1 : 0;
+        ready = __shfl_sync(0xffffffffu, ready, 0);
+        if (ready) {
+          if (lane == 0) {
+            // the other CTAs' stores (generic proxy, acquired above) are read by the copy engine
+            asm volatile("fence.proxy.async;" ::: "memory");
+            const uint32_t bytes = static_cast<uint32_t>(cw.nact) * NPAD * 8;
+            mbar_arrive_expect_tx(&bars->coll_full, bytes);
+            bulk_load(collected, p.partial + static_cast<size_t>(cw.stat) * ncta * NPAD, bytes, &bars->coll_full);
+          }
+          ++cu;
+          do have_c = next_phase(p, cit, cta, ncta, cw); while (have_c && cw.n == 0);
+          progress = true;
+        }
       }
-      ++u;
+      if (progress) {
+        t0 = clock64();
+        spins = 0;
+      } else if ((++spins & 0x3Fu) == 0 && ok) {
+        int give_up = 0;
+        if (lane == 0) {
+          if (*abort_flag) give_up = 1;
+          else if (clock64() - t0 > limit) {
+            *abort_flag = 1;
+            raise_status(p.hdr, FASTKV_ERR_DEVICE_TIMEOUT, have_c && cu < pu ? SITE_FUSED_FLAG : SITE_PARKED_STATS);
+            give_up = 1;
+          }
+        }
+        if (__shfl_sync(0xffffffffu, give_up, 0)) ok = false;
+      }
     }
+    // the last collection issued has landed before the CTA ends, whether pass 2 consumed it or not
+    if (lane == 0 && cu > 0) mbar_wait_drain(&bars->coll_full, (cu - 1) & 1, p.hdr, SITE_PARKED_DRAIN, limit);
   } else if (warp < kCtrlWarps + kPass1Warps) {
     // ---------------- pass 1: logits -> e = exp2(s - ref), row sums ----------------
     // warp (quarter, half) owns tensor-memory lanes 32 * quarter .. +31 (one key per lane) and the
@@ -470,26 +557,34 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     while (next_phase(p, pit, cta, ncta, w)) {           // an aborted CTA still walks every phase: see pass2_sync
       if (w.n == 0) continue;
       const int buf = u & 1;
-      // every CTA that owns tiles of this phase has published its statistics?
-      if (pt == 0 && !*abort_flag) {
-        const int* ctr = p.counters + w.stat;
-        const int target = w.nact + p.extra_publications;
-        if (ld_acquire(ctr) < target) {
-          const long long t0 = clock64();
-          unsigned spins = 0;
-          while (ld_acquire(ctr) < target) {
-            if ((++spins & 0x3Fu) == 0 && (*abort_flag || clock64() - t0 > limit)) {
-              *abort_flag = 1;
-              raise_status(p.hdr, FASTKV_ERR_DEVICE_TIMEOUT, SITE_FUSED_FLAG);
-              break;
+      if (Cfg::kCollect) {
+        // all CTAs' statistics of the phase are in shared memory (the publisher warp saw to it)
+        // (twice the limit: a publication that never comes is reported by the collector, which watches for it)
+        if (ok) ok = mbar_wait_bounded(&bars->coll_full, u & 1, abort_flag, p.hdr, SITE_PARKED_NORM, 2 * limit);
+        const int n2 = 2 * (pt % kTPL), part = pt / kTPL;
+        float2 r0, r1;
+        merge_collected_2rows(collected, NPAD, n2, part, kParts, w.nact, r0, r1);
+        merge_buf[part * NPAD + n2] = r0;
+        merge_buf[part * NPAD + n2 + 1] = r1;
+      } else {
+        // every CTA that owns tiles of this phase has published its statistics?
+        if (pt == 0 && !*abort_flag) {
+          const int* ctr = p.counters + w.stat;
+          const int target = w.nact + p.extra_publications;
+          if (ld_acquire(ctr) < target) {
+            const long long t0 = clock64();
+            unsigned spins = 0;
+            while (ld_acquire(ctr) < target) {
+              if ((++spins & 0x3Fu) == 0 && (*abort_flag || clock64() - t0 > limit)) {
+                *abort_flag = 1;
+                raise_status(p.hdr, FASTKV_ERR_DEVICE_TIMEOUT, SITE_FUSED_FLAG);
+                break;
+              }
             }
           }
         }
-      }
-      pass2_sync();
-      if (*abort_flag) ok = false;
-      // the softmax normaliser of the phase, merged in a fixed order (the same in every CTA)
-      {
+        pass2_sync();
+        // the softmax normaliser of the phase, merged in a fixed order (the same in every CTA)
         const int n2 = 2 * (pt % kTPL), part = pt / kTPL;
         float2 r0, r1;
         merge_partials_2rows(p.partial + static_cast<size_t>(w.stat) * ncta * NPAD, NPAD, n2, part, kParts, w.nact, r0, r1);
@@ -497,6 +592,8 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         merge_buf[part * NPAD + n2 + 1] = r1;
       }
       pass2_sync();
+      if (*abort_flag) ok = false;
+      if (Cfg::kCollect && pt == 0) mbar_arrive(&bars->coll_free);   // the buffer may take the next phase
       if (pt < NPAD) {
         float mm = -INFINITY, ll = 0.0f;
 #pragma unroll
