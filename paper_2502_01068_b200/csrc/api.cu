@@ -386,8 +386,8 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
     const bool parked = lay.path == PATH_PARKED;
     if (parked && parked_tiles_per_cta(s.max_len, ctas) > parked_slots(lay.npad))
       return fail(FASTKV_ERR_UNSUPPORTED, "this device has too few SMs to park a phase of this length");
-    e = cudaMemsetAsync(ws, 0, lay.f_zero_bytes, stream);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace header)");
+    e = parked ? launch_clear_words(ws, lay.f_zero_bytes, stream) : cudaMemsetAsync(ws, 0, lay.f_zero_bytes, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "clearing the workspace header");
     FusedParams fp;
     fp.batch = s.batch; fp.total_len = s.total_len; fp.n_kv_heads = s.n_kv_heads; fp.group = G;
     fp.window = s.window; fp.n_rows = G * s.window; fp.q_layout = s.q_layout;

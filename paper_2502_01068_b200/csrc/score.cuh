@@ -76,6 +76,8 @@ cudaError_t launch_score_fused(int head_dim, int npad, const CUtensorMap& tmap_k
 cudaError_t launch_score_parked(int head_dim, int npad, const CUtensorMap& tmap_k, const CUtensorMap& tmap_q,
                                 const FusedParams& p, int grid, cudaStream_t stream);
 int parked_slots(int npad);   // tiles of one phase a CTA can park: its tiles per phase must not exceed this
+// zeroes `bytes` (a multiple of 4) at `ptr` with a kernel that takes part in the chain of programmatic launches
+cudaError_t launch_clear_words(void* ptr, size_t bytes, cudaStream_t stream);
 cudaError_t launch_pool_rows(const PoolRowsParams& p, int max_len, int batch, cudaStream_t stream);
 
 cudaError_t launch_score_logits(int head_dim, int npad, const CUtensorMap& tmap_k,

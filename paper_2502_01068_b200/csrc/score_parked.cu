@@ -13,19 +13,16 @@
 //              (16 slots of 32 columns, or 8 of 64); a slot is not recycled by the issuer, it is
 //              handed back by pass 2;
 //   pass 1     (eight warps, one key per lane) reads each new slot, turns every logit into
-//              e = exp2(s - ref) against the thread's own reference for that query row, adds e to
-//              the row's running sum and writes e back over the logit; at the end of the phase the
-//              thread's references and the warp's (max, sum) per row go to shared memory.  The
-//              reference of a row is the first logit the thread saw; it moves (and the e already
-//              parked for this phase are rescaled) only if a logit exceeds it by more than 64
-//              binary orders of magnitude;
+//              e = exp2(s - ref) against the warp's reference for that query row, adds e to the
+//              thread's running sum of the row and writes e back over the logit; at the
+//              end of the phase the warp's references and its (reference, sum) per row go to shared
+//              memory.  The reference of a row is the largest logit of the warp's first tile; it
+//              moves (and the e already parked for this phase are rescaled) only if a logit exceeds
+//              it by more than 64 binary orders of magnitude;
 //   publisher  (one warp) writes the CTA's (max, sum) per row of a finished phase to global memory and
-//              bumps the phase's counter, so that publication never waits behind anything else; between
-//              publications it watches the counter of the oldest phase not yet collected and, once
-//              every CTA has published, brings all CTAs' statistics of that phase into shared memory
-//              with one bulk copy -- while pass 2 is still busy with the phase before;
-//   pass 2     (four warps, one per tensor-memory lane quarter) waits for the collected statistics
-//              of the phase, merges them in a fixed order (identical in every CTA:
+//              bumps the phase's counter, so that publication never waits behind anything else;
+//   pass 2     (four warps, one per tensor-memory lane quarter) waits until every CTA of the phase
+//              has published, merges the statistics in a fixed order (identical in every CTA:
 //              deterministic) into the softmax normaliser of every row, forms one weight per
 //              (key lane, query row), f = exp2(ref - M_r) / l_r, and then only needs a multiply-add
 //              per parked value: the score of a key is the sum of e * f over its window rows and
@@ -58,7 +55,7 @@ constexpr int kPass2Threads = 32 * kPass2Warps;
 constexpr int kParkedThreads = 32 * (kCtrlWarps + kPass1Warps + kPass2Warps);   // 15 warps: at most 4 per scheduler
 constexpr int kMaxStages = 8;
 constexpr int kMaxSlots = 16;
-constexpr int kMaxCtas = 148;                  // CTAs whose statistics the collection buffer holds
+constexpr int kRefBufs = 4;                    // phases whose references may be waiting for pass 2
 // Pass 1 keeps e = exp2(s - ref) with the row's first logit as the reference; the reference only moves
 // when a logit exceeds it by more than this many binary orders of magnitude (e and its row sums stay far
 // inside the fp32 range: e <= 2^64, at most 2^20-odd terms per sum).
@@ -69,17 +66,13 @@ struct ParkedCfg {
   static constexpr int KH = D / 64;
   static constexpr int kStageBytes = KH * kHalfBytes;
   static constexpr int kQBytes = KH * NPAD * 128;
-  static constexpr int kStages = (D == 128) ? 3 : 6;
-  // with 32 query rows all CTAs' statistics of a phase (37 KB) are collected in shared memory by the
-  // publisher warp; with 64 rows there is no room and pass 2 reads them from global memory itself
-  static constexpr bool kCollect = NPAD == 32;
-  static constexpr int kCollectBytes = kCollect ? kMaxCtas * NPAD * 8 : 0;
+  static constexpr int kStages = (D == 128) ? 5 : 8;
   static constexpr int kSlots = 512 / NPAD;                 // tensor memory: 512 columns
   static constexpr int kBarBytes = 1024;
-  static constexpr int kRefBytes = NPAD * kTileKeys * 4;    // one reference per (query row, key lane)
-  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 2 * kQBytes + 2 * kRefBytes + kBarBytes +
+  static constexpr int kRefBytes = kRefBufs * 4 * NPAD * 4; // one reference per (phase in flight, lane quarter, query row)
+  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 2 * kQBytes + kRefBytes + kBarBytes +
                                     2 * 4 * NPAD * 8 /*warp_stats*/ + NPAD * 8 /*norm*/ +
-                                    2 * kPass2Threads * 8 /*merge_buf*/ + NPAD * 4 /*row_j*/ + kCollectBytes;
+                                    2 * kPass2Threads * 8 /*merge_buf*/ + NPAD * 4 /*row_j*/;
 };
 
 struct ParkedBarriers {
@@ -87,11 +80,9 @@ struct ParkedBarriers {
   uint64_t q_full[2], q_empty[2];
   uint64_t slot_full[kMaxSlots], slot_free[kMaxSlots];
   uint64_t mma_done;
-  uint64_t ref_free[2];        // pass 2 has finished with the references of a phase
+  uint64_t ref_free[kRefBufs]; // pass 2 has finished with the references of a phase
   uint64_t stats_ready[2];     // pass 1 has written its warps' statistics of a phase
   uint64_t stats_free[2];      // ... and the publisher has read them
-  uint64_t coll_full;          // all CTAs' statistics of a phase have landed in shared memory
-  uint64_t coll_free;          // ... and pass 2 has merged them
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -125,25 +116,20 @@ __device__ __forceinline__ void merge_partials_2rows(const float2* part, int npa
   out1 = make_float2(m1, l1);
 }
 
-// The same merge from the copy of all CTAs' statistics in shared memory.
-__device__ __forceinline__ void merge_collected_2rows(const float2* part, int npad, int n2, int first, int stride,
-                                                      int count, float2& out0, float2& out1) {
-  float m0 = -INFINITY, l0 = 0.0f, m1 = -INFINITY, l1 = 0.0f;
-  for (int r = first; r < count; r += stride) {
-    const float4 v = *reinterpret_cast<const float4*>(&part[r * npad + n2]);
-    merge_stats(m0, l0, v.x, v.y);
-    merge_stats(m1, l1, v.z, v.w);
+// Sums of sixteen values per lane over the 32 lanes of a warp: fifteen exchanges that halve the rows a
+// lane holds, then one between lanes r and r + 16; afterwards both hold the sum of row r in v[0].
+__device__ __forceinline__ void transpose_sum16(float* v, int lane) {
+#pragma unroll
+  for (int o = 8; o >= 1; o >>= 1) {
+    const bool upper = (lane & o) != 0;
+#pragma unroll
+    for (int i = 0; i < o; ++i) {
+      const float send = upper ? v[i] : v[i + o];
+      const float keep = upper ? v[i + o] : v[i];
+      v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+    }
   }
-  out0 = make_float2(m0, l0);
-  out1 = make_float2(m1, l1);
-}
-
-// global -> shared bulk copy (16-byte aligned, size a multiple of 16) that completes on an mbarrier
-__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(smem_dst)),
-               "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
+  v[0] += __shfl_xor_sync(0xffffffffu, v[0], 16);
 }
 
 template <int GG>
@@ -196,13 +182,12 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                                              ~static_cast<uintptr_t>(1023));
   uint8_t* smem_k = smem;
   uint8_t* smem_q = smem_k + kStages * Cfg::kStageBytes;              // two buffers of kQBytes
-  float* smem_ref = reinterpret_cast<float*>(smem_q + 2 * Cfg::kQBytes);   // [2][NPAD][128]: pass 1's references
-  ParkedBarriers* bars = reinterpret_cast<ParkedBarriers*>(smem_q + 2 * Cfg::kQBytes + 2 * Cfg::kRefBytes);
+  float* smem_ref = reinterpret_cast<float*>(smem_q + 2 * Cfg::kQBytes);   // [kRefBufs][4][NPAD]: pass 1's references
+  ParkedBarriers* bars = reinterpret_cast<ParkedBarriers*>(reinterpret_cast<uint8_t*>(smem_ref) + Cfg::kRefBytes);
   float2* warp_stats = reinterpret_cast<float2*>(reinterpret_cast<uint8_t*>(bars) + Cfg::kBarBytes);   // [2][4][NPAD]
   float2* norm = warp_stats + 2 * 4 * NPAD;                           // [NPAD] (-row max, 1 / row sum)
   float2* merge_buf = norm + NPAD;                                    // [256] partial merges
   int* row_j = reinterpret_cast<int*>(merge_buf + 2 * kPass2Threads); // [NPAD] window row j = n / G of query row n
-  float2* collected = reinterpret_cast<float2*>(row_j + NPAD);        // [CTAs][NPAD] (16-byte aligned)
   constexpr int CPW = NPAD / 2;                                       // accumulator columns per pass-1 warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -210,7 +195,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
   const long long limit = p.wait_limit;
 
   // A phase that does not fit in the slot ring could never complete: refuse before any barrier exists.
-  if ((((p.max_len + kTileKeys - 1) / kTileKeys) + ncta - 1) / ncta > kSlots || ncta > kMaxCtas) {
+  if ((((p.max_len + kTileKeys - 1) / kTileKeys) + ncta - 1) / ncta > kSlots) {
     if (cta == 0 && threadIdx.x == 0) raise_status(p.hdr, FASTKV_ERR_UNSUPPORTED, SITE_PARKED_RING);
     return;
   }
@@ -223,13 +208,11 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
       mbar_init(&bars->slot_free[i], kPass2Warps);   // every pass-2 warp reads its lane quarter of the slot
     }
     mbar_init(&bars->mma_done, 1);
+    for (int i = 0; i < kRefBufs; ++i) mbar_init(&bars->ref_free[i], kPass2Warps);
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&bars->ref_free[i], kPass2Warps);
       mbar_init(&bars->stats_ready[i], kPass1Warps);
       mbar_init(&bars->stats_free[i], 1);
     }
-    mbar_init(&bars->coll_full, 1);
-    mbar_init(&bars->coll_free, 1);
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -247,6 +230,10 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
   const uint32_t tmem_base = bars->tmem_base;
   volatile int* abort_flag = &bars->abort_flag;
   pdl_launch_dependents();     // the pooling kernel may be brought up; it waits for this grid to finish
+  // Everything above overlapped the end of the kernel before this one in the stream (the launch allows it);
+  // from here on global memory is read and written: K and Q, the counters the clearing kernel zeroed, and
+  // the un-pooled scores the previous call's pooling kernel may still be reading.
+  pdl_wait();
 
   if (warp == 0) {
     // ---------------- producer: K tiles (and the phase's query rows) by TMA ----------------
@@ -330,88 +317,36 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
       }
     }
   } else if (warp == 2) {
-    // ---------------- publisher: this CTA's row statistics of each finished phase go to global memory; ----------------
-    // ---------------- collector: all CTAs' statistics of a complete phase come back into shared memory ----------------
-    // Two walks over the phase list, `pw` for publication and `cw` for collection; whichever has something to
-    // do goes first, so a publication never waits behind a collection and the other way round.
-    int pu = 0, cu = 0;                                  // phases with tiles here: published / collected
+    // ---------------- publisher: this CTA's row statistics of each finished phase go to global memory ----------------
+    int u = 0;
     bool ok = true;
-    PhaseIter pit = {0, 0}, cit = {0, 0};
-    PhaseWork pw, cw;
-    bool have_p = next_phase(p, pit, cta, ncta, pw), have_c = Cfg::kCollect && next_phase(p, cit, cta, ncta, cw);
-    while (have_p && pw.n == 0) have_p = next_phase(p, pit, cta, ncta, pw);
-    while (have_c && cw.n == 0) have_c = next_phase(p, cit, cta, ncta, cw);
-    long long t0 = clock64();
-    unsigned spins = 0;
-    while (have_p || have_c) {
-      bool progress = false;
-      if (have_p) {
-        const int buf = pu & 1;
-        int ready = 1;
-        if (ok && lane == 0) ready = mbar_try_wait(&bars->stats_ready[buf], (pu >> 1) & 1) ? 1 : 0;
-        ready = __shfl_sync(0xffffffffu, ready, 0);
-        if (ready) {                                     // (an aborted CTA publishes without waiting: nobody hangs on it)
-          __syncwarp();
-          const float2* ws = warp_stats + buf * 4 * NPAD;
+    PhaseIter pit = {0, 0};
+    PhaseWork w;
+    while (next_phase(p, pit, cta, ncta, w)) {
+      if (w.n == 0) continue;
+      const int buf = u & 1;
+      if (ok) ok = mbar_wait_bounded(&bars->stats_ready[buf], (u >> 1) & 1, abort_flag, p.hdr, SITE_PARKED_STATS, limit);
+      ok = __all_sync(0xffffffffu, ok);
+      const float2* ws = warp_stats + buf * 4 * NPAD;
 #pragma unroll
-          for (int n = lane; n < NPAD; n += 32) {        // lane quarters -> CTA
-            float mm = -INFINITY, ll = 0.0f;
+      for (int n = lane; n < NPAD; n += 32) {            // lane quarters -> CTA
+        float mm = -INFINITY, ll = 0.0f;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) merge_stats(mm, ll, ws[q * NPAD + n].x, ws[q * NPAD + n].y);
-            p.partial[(static_cast<size_t>(pw.stat) * ncta + cta) * NPAD + n] = make_float2(mm, ll);
-          }
-          __syncwarp();
-          if (lane == 0) {
-            red_release_add(p.counters + pw.stat, 1);    // release: cumulative over the warp's stores
-            mbar_arrive(&bars->stats_free[buf]);
-          }
-          ++pu;
-          do have_p = next_phase(p, pit, cta, ncta, pw); while (have_p && pw.n == 0);
-          progress = true;
-        }
+        for (int q = 0; q < 4; ++q) merge_stats(mm, ll, ws[q * NPAD + n].x, ws[q * NPAD + n].y);
+        p.partial[(static_cast<size_t>(w.stat) * ncta + cta) * NPAD + n] = make_float2(mm, ll);
       }
-      if (have_c && !ok) have_c = false;                 // aborted: nothing more is collected
-      if (have_c && cu < pu) {
-        int ready = 0;
-        if (lane == 0)                                   // the buffer is free again and every CTA has published?
-          ready = (mbar_try_wait(&bars->coll_free, (cu & 1) ^ 1) &&
-                   ld_acquire(p.counters + cw.stat) >= cw.nact + p.extra_publications) ? 1 : 0;
-        ready = __shfl_sync(0xffffffffu, ready, 0);
-        if (ready) {
-          if (lane == 0) {
-            // the other CTAs' stores (generic proxy, acquired above) are read by the copy engine
-            asm volatile("fence.proxy.async;" ::: "memory");
-            const uint32_t bytes = static_cast<uint32_t>(cw.nact) * NPAD * 8;
-            mbar_arrive_expect_tx(&bars->coll_full, bytes);
-            bulk_load(collected, p.partial + static_cast<size_t>(cw.stat) * ncta * NPAD, bytes, &bars->coll_full);
-          }
-          ++cu;
-          do have_c = next_phase(p, cit, cta, ncta, cw); while (have_c && cw.n == 0);
-          progress = true;
-        }
+      __syncwarp();
+      if (lane == 0) {
+        red_release_add(p.counters + w.stat, 1);         // release: cumulative over the warp's stores
+        mbar_arrive(&bars->stats_free[buf]);
       }
-      if (progress) {
-        t0 = clock64();
-        spins = 0;
-      } else if ((++spins & 0x3Fu) == 0 && ok) {
-        int give_up = 0;
-        if (lane == 0) {
-          if (*abort_flag) give_up = 1;
-          else if (clock64() - t0 > limit) {
-            *abort_flag = 1;
-            raise_status(p.hdr, FASTKV_ERR_DEVICE_TIMEOUT, have_c && cu < pu ? SITE_FUSED_FLAG : SITE_PARKED_STATS);
-            give_up = 1;
-          }
-        }
-        if (__shfl_sync(0xffffffffu, give_up, 0)) ok = false;
-      }
+      ++u;
     }
-    // the last collection issued has landed before the CTA ends, whether pass 2 consumed it or not
-    if (lane == 0 && cu > 0) mbar_wait_drain(&bars->coll_full, (cu - 1) & 1, p.hdr, SITE_PARKED_DRAIN, limit);
   } else if (warp < kCtrlWarps + kPass1Warps) {
     // ---------------- pass 1: logits -> e = exp2(s - ref), row sums ----------------
     // warp (quarter, half) owns tensor-memory lanes 32 * quarter .. +31 (one key per lane) and the
-    // accumulator columns (query rows) half * CPW .. +CPW-1.
+    // accumulator columns (query rows) half * CPW .. +CPW-1.  The reference m[] of a row is the same in
+    // all lanes of the warp; the sums l[] are the thread's own.
     const int gw = warp - kCtrlWarps;
     const int quarter = warp & 3, half = gw >> 2;
     const int key_in_tile = quarter * 32 + lane;
@@ -429,7 +364,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
           raise_status(p.hdr, FASTKV_ERR_INVALID_ARG, SITE_SCORE_SHORT_SEQUENCE);
         continue;
       }
-      float m[CPW], l[CPW];                              // this thread's reference and sum of e per query row
+      float m[CPW], l[CPW];                              // the warp's reference and this thread's sum of e per query row
 #pragma unroll
       for (int n = 0; n < CPW; ++n) { m[n] = -INFINITY; l[n] = 0.0f; }
       const int win_start = w.L - p.window;
@@ -449,9 +384,34 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
           const int n_valid = n_rows - col0 - c * 16;
           float* const mc = m + c * 16;
           float* const lc = l + c * 16;
-          bool general = !tile_unmasked || i == 0;
-          if (!general) {
-            // common case: no logit is far above its reference, one exp2 per logit and nothing else
+          bool general = !tile_unmasked;
+          if (!general && i == 0) {
+            // first tile of the phase, every key visible: lane 0's logit starts the row's reference
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+              const float first = __shfl_sync(0xffffffffu, v[r] * p.scale_log2, 0);
+              if (r < n_valid) mc[r] = first;
+            }
+          }
+          if (!general && n_valid >= 16) {
+            // common case: every row in use, no logit far above its reference: one multiply-add, one exp2
+            // and one add per logit, and a maximum to find out
+            float x[16];
+#pragma unroll
+            for (int r = 0; r < 16; ++r) x[r] = fmaf(v[r], p.scale_log2, -mc[r]);
+            const float top = fmaxf(fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7]))),
+                                    fmaxf(fmaxf(fmaxf(x[8], x[9]), fmaxf(x[10], x[11])), fmaxf(fmaxf(x[12], x[13]), fmaxf(x[14], x[15]))));
+            general = __any_sync(0xffffffffu, top > kRefSlackLog2);
+            if (!general) {
+#pragma unroll
+              for (int r = 0; r < 16; ++r) {
+                const float e = ex2(x[r]);
+                lc[r] += e;
+                v[r] = e;
+              }
+            }
+          } else if (!general) {
+            // the same with unused (padding) rows among the sixteen
             float x[16];
             bool far = false;
 #pragma unroll
@@ -470,8 +430,8 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             }
           }
           if (general) {
-            // first tile of the phase, a tile that overlaps the observation window (causal mask), or a
-            // logit far above its reference: per row, start / keep / move the reference
+            // a tile that overlaps the observation window (causal mask), or a logit far above its reference:
+            // per row, start / keep / move the warp's reference
             uint32_t visible = 0xFFFFu;
             if (!tile_unmasked) {
               visible = 0;
@@ -481,30 +441,36 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                   if (r < n_valid && key <= win_start + row_j[col0 + c * 16 + r]) visible |= 1u << r;
               }
             }
+            float sl[16], xm[16];
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+              sl[r] = (r < n_valid && ((visible >> r) & 1u)) ? v[r] * p.scale_log2 : -INFINITY;
+              xm[r] = sl[r];
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) {
+#pragma unroll
+              for (int r = 0; r < 16; ++r) xm[r] = fmaxf(xm[r], __shfl_xor_sync(0xffffffffu, xm[r], off));
+            }
             float fac[16];
-            bool moved = false;
+            bool moved = false;                          // the same in every lane: xm and mc are
 #pragma unroll
             for (int r = 0; r < 16; ++r) {
               fac[r] = 1.0f;
-              if (r >= n_valid || !((visible >> r) & 1u)) { v[r] = 0.0f; continue; }
-              const float sl = v[r] * p.scale_log2;
-              if (mc[r] == -INFINITY) {                  // first logit of the row: it becomes the reference
-                mc[r] = sl; lc[r] = 1.0f; v[r] = 1.0f;
-              } else {
-                const float x = sl - mc[r];
-                if (x > kRefSlackLog2) {                 // move the reference up to this logit
-                  fac[r] = ex2(-x);
-                  lc[r] = lc[r] * fac[r] + 1.0f;
-                  mc[r] = sl; v[r] = 1.0f;
-                  moved = true;
-                } else {
-                  const float e = ex2(x);
-                  lc[r] += e;
-                  v[r] = e;
-                }
+              if (xm[r] == -INFINITY) { v[r] = 0.0f; continue; }     // nothing of this row is visible to the warp here
+              if (mc[r] == -INFINITY) {
+                mc[r] = xm[r];                           // first logits of the row: the largest becomes the reference
+              } else if (xm[r] - mc[r] > kRefSlackLog2) {            // move the reference up
+                fac[r] = ex2(mc[r] - xm[r]);
+                lc[r] *= fac[r];
+                mc[r] = xm[r];
+                moved = true;
               }
+              const float e = ex2(sl[r] - mc[r]);        // exp2(-inf) = 0 for a masked key
+              lc[r] += e;
+              v[r] = e;
             }
-            if (__any_sync(0xffffffffu, moved)) {        // rescale what this warp parked earlier in the phase
+            if (moved) {                                 // rescale what this warp parked earlier in the phase
               tmem_wait_st();
               for (int Tp = T0; Tp < T; ++Tp) {
                 float old[16];
@@ -519,20 +485,26 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
           tmem_st_32x16(lane_base + a * NPAD + c * 16, v);
         }
       }
-      // this thread's references go to pass 2, the warp's (max, sum) per row to the statistics group, as
-      // soon as they are done with the buffers of the phase before last
-      const int buf = u & 1;
+      // the warp's references go to pass 2, its (reference, sum) per row to the publisher, as soon as
+      // they are done with the buffers of earlier phases
+      const int buf = u & 1, rbuf = u % kRefBufs;
+      if (ok && u >= kRefBufs)
+        ok = mbar_wait_bounded(&bars->ref_free[rbuf], ((u / kRefBufs) - 1) & 1, abort_flag, p.hdr, SITE_PARKED_REF, limit);
       if (ok && u >= 2)
-        ok = mbar_wait_bounded(&bars->ref_free[buf], ((u >> 1) - 1) & 1, abort_flag, p.hdr, SITE_PARKED_REF, limit) &&
-             mbar_wait_bounded(&bars->stats_free[buf], ((u >> 1) - 1) & 1, abort_flag, p.hdr, SITE_PARKED_STATS, limit);
-      float* const ref_out = smem_ref + (buf * NPAD + col0) * kTileKeys + key_in_tile;
+        ok = mbar_wait_bounded(&bars->stats_free[buf], ((u >> 1) - 1) & 1, abort_flag, p.hdr, SITE_PARKED_STATS, limit);
+      float* const ref_out = smem_ref + (rbuf * 4 + quarter) * NPAD + col0;
+      if (lane == 0) {
 #pragma unroll
-      for (int n = 0; n < CPW; ++n) ref_out[n * kTileKeys] = m[n];
-      // lanes -> warp: after the butterfly lanes r and r + 16 hold row col0 + c * 16 + r in entry c * 16
+        for (int n = 0; n < CPW; ++n) ref_out[n] = m[n];
+      }
+      __syncwarp();
+      // lanes -> warp: the reference of a row is the same in all lanes, so its sums just add up; after
+      // the butterfly lanes r and r + 16 hold the sum of row col0 + c * 16 + r in entry c * 16
 #pragma unroll
       for (int c = 0; c < CPW / 16; ++c) {
-        stats_transpose_merge<16>(m + c * 16, l + c * 16, lane);
-        if (lane < 16) warp_stats[(buf * 4 + quarter) * NPAD + col0 + c * 16 + lane] = make_float2(m[c * 16], l[c * 16]);
+        transpose_sum16(l + c * 16, lane);
+        if (lane < 16)
+          warp_stats[(buf * 4 + quarter) * NPAD + col0 + c * 16 + lane] = make_float2(ref_out[c * 16 + lane], l[c * 16]);
       }
       tmem_wait_st();                                    // the parked e are read by pass 2 once the statistics are merged
       tc_fence_before_sync();
@@ -556,17 +528,8 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     PhaseWork w;
     while (next_phase(p, pit, cta, ncta, w)) {           // an aborted CTA still walks every phase: see pass2_sync
       if (w.n == 0) continue;
-      const int buf = u & 1;
-      if (Cfg::kCollect) {
-        // all CTAs' statistics of the phase are in shared memory (the publisher warp saw to it)
-        // (twice the limit: a publication that never comes is reported by the collector, which watches for it)
-        if (ok) ok = mbar_wait_bounded(&bars->coll_full, u & 1, abort_flag, p.hdr, SITE_PARKED_NORM, 2 * limit);
-        const int n2 = 2 * (pt % kTPL), part = pt / kTPL;
-        float2 r0, r1;
-        merge_collected_2rows(collected, NPAD, n2, part, kParts, w.nact, r0, r1);
-        merge_buf[part * NPAD + n2] = r0;
-        merge_buf[part * NPAD + n2 + 1] = r1;
-      } else {
+      const int rbuf = u % kRefBufs;
+      {
         // every CTA that owns tiles of this phase has published its statistics?
         if (pt == 0 && !*abort_flag) {
           const int* ctr = p.counters + w.stat;
@@ -593,7 +556,6 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
       }
       pass2_sync();
       if (*abort_flag) ok = false;
-      if (Cfg::kCollect && pt == 0) mbar_arrive(&bars->coll_free);   // the buffer may take the next phase
       if (pt < NPAD) {
         float mm = -INFINITY, ll = 0.0f;
 #pragma unroll
@@ -603,20 +565,20 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
       }
       pass2_sync();
       tc_fence_after_sync();
-      // one weight per query row for this thread's key lane: f = exp2(ref - M) / l (ref = -inf: nothing parked)
-      float* const ref_in = smem_ref + (buf * NPAD) * kTileKeys + key_in_tile;
+      // one weight per query row for this warp's keys: f = exp2(ref - M) / l (ref = -inf: nothing parked)
+      float* const ref_in = smem_ref + (rbuf * 4 + quarter) * NPAD;
       float f[NPAD == 32 ? 32 : 1];
       if (NPAD == 32) {
+        const float2 st = norm[lane];
+        const float mine = ex2(ref_in[lane] + st.x) * st.y;
 #pragma unroll
-        for (int r = 0; r < 32; ++r) {
+        for (int r = 0; r < 32; ++r) f[r] = __shfl_sync(0xffffffffu, mine, r);
+      } else {                                           // many rows: the weights replace the warp's references
+        for (int r = lane; r < NPAD; r += 32) {
           const float2 st = norm[r];
-          f[r] = ex2(ref_in[r * kTileKeys] + st.x) * st.y;
+          ref_in[r] = ex2(ref_in[r] + st.x) * st.y;
         }
-      } else {                                           // many rows: the weights replace this thread's references
-        for (int r = 0; r < NPAD; ++r) {
-          const float2 st = norm[r];
-          ref_in[r * kTileKeys] = ex2(ref_in[r * kTileKeys] + st.x) * st.y;
-        }
+        __syncwarp();
       }
       for (int i = 0; i < w.n; ++i, ++T) {
         const int a = T % kSlots;
@@ -638,13 +600,20 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->slot_free[a]);
           }
-#pragma unroll
-          for (int x = 0; x < 32; ++x)
-            pr[x] *= (NPAD == 32) ? f[x % (NPAD == 32 ? 32 : 1)] : ref_in[(c * 32 + x) * kTileKeys];
           if (!p.per_head) {
+            float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;      // four chains of multiply-adds, fixed order
 #pragma unroll
-            for (int x = 0; x < 32; x += 4) a_g += (pr[x] + pr[x + 1]) + (pr[x + 2] + pr[x + 3]);
+            for (int x = 0; x < 32; x += 4) {
+              s0 = fmaf(pr[x], (NPAD == 32) ? f[x % (NPAD == 32 ? 32 : 1)] : ref_in[c * 32 + x], s0);
+              s1 = fmaf(pr[x + 1], (NPAD == 32) ? f[(x + 1) % (NPAD == 32 ? 32 : 1)] : ref_in[c * 32 + x + 1], s1);
+              s2 = fmaf(pr[x + 2], (NPAD == 32) ? f[(x + 2) % (NPAD == 32 ? 32 : 1)] : ref_in[c * 32 + x + 2], s2);
+              s3 = fmaf(pr[x + 3], (NPAD == 32) ? f[(x + 3) % (NPAD == 32 ? 32 : 1)] : ref_in[c * 32 + x + 3], s3);
+            }
+            a_g += (s0 + s1) + (s2 + s3);
           } else {                                       // row n = j * G + hl and G divides 32
+#pragma unroll
+            for (int x = 0; x < 32; ++x)
+              pr[x] *= (NPAD == 32) ? f[x % (NPAD == 32 ? 32 : 1)] : ref_in[c * 32 + x];
             switch (G) {
               case 1: add_heads<1>(pr, a_h); break;
               case 2: add_heads<2>(pr, a_h); break;
@@ -664,7 +633,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         }
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->ref_free[buf]);  // pass 1 may overwrite this phase's references
+      if (lane == 0) mbar_arrive(&bars->ref_free[rbuf]); // pass 1 may overwrite this phase's references
       pass2_sync();                                      // norm / merge_buf are rewritten next phase
       ++u;
     }
@@ -684,6 +653,27 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 
 int parked_slots(int npad) { return 512 / npad; }
 
+// Zeroes the workspace header and the phase counters ahead of the scoring kernel.  A kernel rather than a
+// memset so that it can sit in the chain of programmatic launches: it comes up while the kernel before it
+// is still running and lets the scoring kernel come up behind it.
+__global__ void clear_words_kernel(uint32_t* words, int n) {
+  pdl_launch_dependents();
+  pdl_wait();
+  for (int i = threadIdx.x; i < n; i += blockDim.x) words[i] = 0u;
+}
+
+cudaError_t launch_clear_words(void* ptr, size_t bytes, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(1);
+  cfg.blockDim = dim3(256);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  fill_pdl_attribute(&attr[0]);
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, clear_words_kernel, static_cast<uint32_t*>(ptr), static_cast<int>(bytes / 4));
+}
+
 template <int D, int NPAD>
 static cudaError_t launch_parked_t(const CUtensorMap& tk, const CUtensorMap& tq, const FusedParams& p, int grid,
                                    cudaStream_t stream) {
@@ -699,6 +689,27 @@ static cudaError_t launch_parked_t(const CUtensorMap& tk, const CUtensorMap& tq,
     configured.set(dev);
   }
   void* args[] = {const_cast<CUtensorMap*>(&tk), const_cast<CUtensorMap*>(&tq), const_cast<FusedParams*>(&p)};
+  // cooperative (every CTA resident: they wait on one another) and, where the driver takes both attributes
+  // together, programmatic as well: the kernel's set-up then overlaps the end of the kernel before it
+  static PerDeviceOnce no_overlap;
+  if (!no_overlap.done(dev)) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kParkedThreads);
+    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    fill_pdl_attribute(&attr[1]);
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    e = cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(score_parked_kernel<D, NPAD>), args);
+    if (e == cudaSuccess) return e;
+    if (e != cudaErrorNotSupported && e != cudaErrorInvalidValue) return e;
+    cudaGetLastError();          // the combination is refused: from now on plain cooperative launches
+    no_overlap.set(dev);
+  }
   return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(score_parked_kernel<D, NPAD>), dim3(grid),
                                      dim3(kParkedThreads), args, Cfg::kSmemBytes, stream);
 }

@@ -100,25 +100,28 @@ def test_every_scoring_kernel_matches(debug_hooks, path):
             check_layer(wl, x, g, o, what="path %d" % path)
 
 
-def test_sequence_longer_than_half_the_tensor_memory_ring():
+def test_sequence_longer_than_half_the_tensor_memory_ring(debug_hooks):
     """L = 160 000: a CTA would own 9 tiles per phase, more than half of the 16 parked slots, so the
     library picks the kernel that re-reads K from L2 by itself; the parked kernel, forced, still works
     (9 <= 16) and gives the same result up to rounding."""
     wl = small("long", 601, [160000], [4000], [8000], Hq=4, Hkv=1, d=64, hidden=64)
     x = W.make_layer(wl)
-    g = gpu_layer(wl, x)
     o = oracle_layer(wl, x)
-    check_layer(wl, x, g, o, what="160k")
+    check_layer(wl, x, gpu_layer(wl, x), o, what="160k")
+    debug_hooks("score_path", 3)
+    check_layer(wl, x, gpu_layer(wl, x), o, what="160k parked")
 
 
 def test_parked_kernel_at_the_edge_of_its_ring(debug_hooks):
+    """148 CTAs x 16 slots x 128 keys = 303 104 keys is the most the parked kernel can hold per phase:
+    every slot of the ring is in use at once."""
     debug_hooks("score_path", 3)
-    wl = small("long", 601, [160000], [4000], [8000], Hq=4, Hkv=1, d=64, hidden=64)
+    wl = small("edge", 602, [303000], [4000], [8000], Hq=4, Hkv=1, d=64, hidden=64)
     x = W.make_layer(wl)
     g = gpu_layer(wl, x)
     o = oracle_layer(wl, x)
-    check_layer(wl, x, g, o, what="160k parked")
-    # beyond 148 CTAs x 16 slots x 128 keys the parked kernel cannot run: refused on the host
+    check_layer(wl, x, g, o, what="303k parked")
+    # beyond that the parked kernel cannot run: refused on the host
     shape = B.make_shape(total_len=310000, n_q_heads=4, n_kv_heads=1, head_dim=64)
     with pytest.raises(B.FastKVError) as e:
         B.fastkv_workspace_bytes(shape)
