@@ -44,6 +44,7 @@ def _load():
         lib.oracle_select.argtypes = [vp, i64, i64, i32, i32, vp, vp]
         lib.oracle_gather_rows.argtypes = [vp, i64, i64, vp, i64, vp]
         lib.oracle_decode_attention.argtypes = [vp, vp, vp, i64, i32, i32, i32, f64, vp, vp]
+        lib.oracle_prefill_attention.argtypes = [vp, vp, vp, i64, i32, i32, i32, f64, vp]
         lib.oracle_num_threads.restype = i32
         _lib = lib
     return _lib
@@ -154,3 +155,17 @@ def decode_attention(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray, sc
     if rc:
         raise ValueError("oracle_decode_attention rejected its arguments")
     return out, lse
+
+
+def prefill_attention(q_full: np.ndarray, k: np.ndarray, v: np.ndarray, scale: Optional[float] = None) -> np.ndarray:
+    """Causal softmax attention of a whole prompt (the layer's own attention, Alg. 1): q_full [L, H, d],
+    k / v [L, Hkv, d] (bf16 bits).  Returns O [L, H, d] fp64."""
+    q_full, k, v = _u16(q_full), _u16(k), _u16(v)
+    L, H, d = q_full.shape
+    Hkv = k.shape[1]
+    out = np.empty((L, H, d), dtype=np.float64)
+    rc = _load().oracle_prefill_attention(_ptr(q_full), _ptr(k), _ptr(v), L, H, Hkv, d,
+                                          (d ** -0.5) if scale is None else scale, _ptr(out))
+    if rc:
+        raise ValueError("oracle_prefill_attention rejected its arguments")
+    return out

@@ -28,8 +28,8 @@
  * Parity pins (tests/test_oracle_*.py): full LxL causal attention through a
  * library softmax, the uniform-attention and single-planted-key closed forms,
  * row-sum / shift / permutation invariants, pooling identities, selection
- * against a brute-force ranking, gather against numpy indexing, decode attention against a
- * library softmax-attention and closed forms.  Nothing
+ * against a brute-force ranking, gather against numpy indexing, decode and prefill attention
+ * against a library softmax-attention and closed forms.  Nothing
  * numeric from the paper's own implementation exists to compare against, so
  * parity with that implementation is unpinned; parity with the definitions
  * above is pinned.
@@ -299,6 +299,48 @@ int oracle_decode_attention(const uint16_t* q, const uint16_t* k_cache, const ui
     }
     free(s);
     return 0;
+}
+
+/*
+ * The layer's own attention (Alg. 1: X <- layer_l(X) produces Att_l; Sec. 4.2: the saliency scores are read
+ * off that same matrix): the output of causal softmax attention for every query position,
+ *   O[t, h, :] = sum_{i <= t} Att_l[h, t, i] * V[i, h/G, :],
+ *   Att_l[h, t, i] = exp(s_i - max_i' s_i') / sum_i' exp(s_i' - max), s_i = scale * <Q[t,h,:], K[i,h/G,:]>, i <= t.
+ * q is [L, H, d], k and v are [L, Hkv, d] (bf16 bits, dense); O is [L, H, d] fp64.
+ */
+int oracle_prefill_attention(const uint16_t* q, const uint16_t* k, const uint16_t* v, int64_t L, int H, int Hkv,
+                             int d, double scale, double* O) {
+    if (L < 1 || H % Hkv != 0) return 1;
+    const int G = H / Hkv;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int h = 0; h < H; ++h) {
+        const int g = h / G;
+        double* s = (double*)malloc((size_t)L * sizeof(double));
+        if (!s) { failed = 1; continue; }
+        for (int64_t t = 0; t < L; ++t) {
+            const uint16_t* qrow = q + (t * H + h) * (int64_t)d;
+            double smax = -INFINITY;
+            for (int64_t i = 0; i <= t; ++i) {                 /* causal: keys 0..t */
+                const uint16_t* krow = k + (i * Hkv + g) * (int64_t)d;
+                double acc = 0.0;
+                for (int c = 0; c < d; ++c) acc += bf16_to_f64(qrow[c]) * bf16_to_f64(krow[c]);
+                s[i] = scale * acc;
+                if (s[i] > smax) smax = s[i];
+            }
+            double denom = 0.0;
+            for (int64_t i = 0; i <= t; ++i) denom += exp(s[i] - smax);
+            double* out = O + (t * H + h) * (int64_t)d;
+            for (int c = 0; c < d; ++c) out[c] = 0.0;
+            for (int64_t i = 0; i <= t; ++i) {
+                const double p = exp(s[i] - smax) / denom;
+                const uint16_t* vrow = v + (i * Hkv + g) * (int64_t)d;
+                for (int c = 0; c < d; ++c) out[c] += p * bf16_to_f64(vrow[c]);
+            }
+        }
+        free(s);
+    }
+    return failed;
 }
 
 int oracle_num_threads(void) {

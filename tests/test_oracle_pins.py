@@ -341,3 +341,43 @@ def test_decode_attention_matches_library_attention_and_closed_forms():
     out_p, lse_p = oracle.decode_attention(q, kc[:, perm], vc[:, perm])
     np.testing.assert_allclose(out_p, out, rtol=0, atol=1e-13)
     np.testing.assert_allclose(lse_p, lse, rtol=0, atol=1e-13)
+
+
+@pytest.mark.parametrize("L,H,Hkv,d", [(70, 4, 2, 16), (33, 6, 3, 8), (9, 2, 2, 32)])
+def test_prefill_attention_matches_library_attention_and_closed_forms(L, H, Hkv, d):
+    """The layer's own causal attention (whose matrix the saliency scores are read off): pinned against
+    torch's scaled_dot_product_attention in fp64, against the matrix-times-values product of the
+    brute-force attention matrix, and against closed forms."""
+    rng = np.random.default_rng(100 + L)
+    q, k = rand_qk(L + 3, L, H, Hkv, d)
+    v = bf16(rng.standard_normal((L, Hkv, d)))
+    O = oracle.prefill_attention(q, k, v)
+    G = H // Hkv
+    tq = torch.from_numpy(f64(q)).permute(1, 0, 2)[None]                          # [1, H, L, d]
+    tk = torch.from_numpy(f64(k)).repeat_interleave(G, dim=1).permute(1, 0, 2)[None]
+    tv = torch.from_numpy(f64(v)).repeat_interleave(G, dim=1).permute(1, 0, 2)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True)[0].permute(1, 0, 2).numpy()
+    np.testing.assert_allclose(O, ref, rtol=0, atol=1e-13)
+    # the same through the explicit attention matrix (torch.softmax route of the window pin)
+    _, att = torch_window_attention(q, k, 1)                                       # [H, L, L]
+    vv = f64(v).repeat(G, axis=1)                                                  # [L, H, d]
+    np.testing.assert_allclose(O, np.einsum("hti,ihd->thd", att, vv), rtol=0, atol=1e-13)
+    # the first token attends to itself only
+    np.testing.assert_allclose(O[0], vv[0], rtol=0, atol=1e-15)
+    # all value rows equal: the output is that row, whatever the weights
+    v_same = np.broadcast_to(v[:1], v.shape).copy()
+    np.testing.assert_allclose(oracle.prefill_attention(q, k, v_same), np.broadcast_to(vv[:1], O.shape), rtol=0, atol=1e-13)
+    # zero queries: uniform causal weights, the output is the running mean of the values
+    O_u = oracle.prefill_attention(np.zeros_like(q), k, v)
+    run_mean = np.cumsum(vv, axis=0) / np.arange(1, L + 1)[:, None, None]
+    np.testing.assert_allclose(O_u, run_mean, rtol=0, atol=1e-13)
+    # a different scale changes the result the way the definition says (scale 0 = uniform weights)
+    np.testing.assert_allclose(oracle.prefill_attention(q, k, v, scale=1e-30), run_mean, rtol=0, atol=1e-12)
+    # one key far above the rest for every query after it: the output is that key's value row
+    star = L // 3
+    q_hot = np.broadcast_to(q[:1, ::G].repeat(G, axis=1), q.shape).copy()          # every position and every head of a group asks the same
+    k_hot = np.zeros_like(k)
+    k_hot[star] = bf16(60.0 * f64(q)[0, ::G])
+    O_h = oracle.prefill_attention(q_hot, k_hot, v)
+    np.testing.assert_allclose(O_h[star:], np.broadcast_to(vv[star], O_h[star:].shape), rtol=0, atol=1e-9)
+    np.testing.assert_allclose(O_h[:star], run_mean[:star], rtol=0, atol=1e-13)   # before it: all logits are 0
