@@ -175,6 +175,25 @@ int fastkv_decode_attn(const fastkv_shape* shape, const void* q, const void* k_c
                        void* stream);
 
 /*
+ * The layer's own causal attention with the saliency scores as a by-product (Alg. 1: the scores are read off
+ * Att_l, the attention matrix of the layer that is being computed anyway; App. D.4 times the separate
+ * "token importance estimation" pass this call makes unnecessary).  For every sequence b and query head h
+ *   out[t, h, :] = sum_{i <= t} softmax_i(scale * <q[t, h], k[i, h / G]>) * v[i, h / G, :]        t = 0 .. L_b - 1
+ * and, from the rows t = L_b - w .. L_b - 1 of the same attention matrix, the scores fastkv_score defines:
+ *   scores_kv [n_kv_heads, total_len] fp32 (may be NULL: attention only), scores_tsp [total_len] fp32 or NULL.
+ * q: bf16, the FULL packed queries [total_len, n_q_heads, head_dim] (shape->q_layout must be FASTKV_Q_FULL);
+ * k, v: bf16 [total_len, n_kv_heads, head_dim]; strides as in the shape (multiples of 8 elements);
+ * out: bf16, dense [total_len, n_q_heads, head_dim], 16-byte aligned.  Probabilities are rounded to bf16 before
+ * they are multiplied with v (fp32 accumulation), the scores are formed from the fp32 logits.
+ * workspace: >= fastkv_prefill_workspace_bytes, 256-byte aligned: the header with the status word (cleared by this
+ * call), the window rows' logits (n_q_heads x window x total_len fp32) and one un-pooled score row per KV head.
+ */
+int fastkv_prefill_workspace_bytes(const fastkv_shape* shape, size_t* bytes);
+int fastkv_prefill_attention(const fastkv_shape* shape, const void* q, const void* k, const void* v, void* out,
+                             float* scores_kv, float* scores_tsp, void* workspace, size_t workspace_bytes,
+                             void* stream);
+
+/*
  * Synchronises `stream`, then copies the device status word of `workspace` to the HOST
  * integers *status (a fastkv_status) and *site (which wait or check raised it; 0 if none).
  */
@@ -251,7 +270,7 @@ int fastkv_debug_set(const char* key, int64_t value);
 /*
  * Sum of the device durations (HOST double, milliseconds) and number of launches recorded for one
  * kernel class since the last query (0 scoring kernel, 1 pooling kernel, 2 selection, 3 compaction,
- * 4 decode attention); waits for the recorded launches and forgets them.  *name receives a static
+ * 4 decode attention, 5 prefill attention, 6 window scores); waits for the recorded launches and forgets them.  *name receives a static
  * string.  Any of the three outputs may be NULL.  No counterpart in the paper (measurement aid).
  */
 int fastkv_debug_kernel_time(int32_t kernel, double* total_ms, int64_t* launches, const char** name);

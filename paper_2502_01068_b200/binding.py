@@ -21,7 +21,8 @@ GROUP_THEN_POOL, POOL_THEN_GROUP = 0, 1
 Q_FULL, Q_WINDOW = 0, 1
 
 EXPORTS = ["fastkv_workspace_bytes", "fastkv_score", "fastkv_select_kv", "fastkv_select_tsp", "fastkv_select",
-           "fastkv_compact", "fastkv_decode_attn_workspace_bytes", "fastkv_decode_attn", "fastkv_device_status", "fastkv_layer_host_arena_bytes",
+           "fastkv_compact", "fastkv_decode_attn_workspace_bytes", "fastkv_decode_attn", "fastkv_prefill_workspace_bytes",
+           "fastkv_prefill_attention", "fastkv_device_status", "fastkv_layer_host_arena_bytes",
            "fastkv_layer_host", "fastkv_score_static", "fastkv_score_static_status", "fastkv_debug_set",
            "fastkv_debug_kernel_time",
            "fastkv_status_string", "fastkv_last_error", "fastkv_kernel_launches"]
@@ -86,6 +87,8 @@ def _load():
         lib.fastkv_score_static.argtypes = [ps, vp, vp, vp, vp, vp]
         lib.fastkv_decode_attn_workspace_bytes.argtypes = [ps, ctypes.POINTER(sz)]
         lib.fastkv_decode_attn.argtypes = [ps, vp, vp, vp, pb, vp, vp, vp, sz, vp]
+        lib.fastkv_prefill_workspace_bytes.argtypes = [ps, ctypes.POINTER(sz)]
+        lib.fastkv_prefill_attention.argtypes = [ps, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.fastkv_score_static_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
         lib.fastkv_debug_set.argtypes = [ctypes.c_char_p, ctypes.c_int64]
         lib.fastkv_debug_kernel_time.argtypes = [ctypes.c_int32, ctypes.POINTER(ctypes.c_double),
@@ -202,6 +205,18 @@ def fastkv_decode_attn(shape: Shape, q, k_cache, v_cache, kv: Budget, out, lse, 
     _check(_load().fastkv_decode_attn(ctypes.byref(shape), _p(q), _p(k_cache), _p(v_cache), ctypes.byref(kv), _p(out),
                                       _p(lse), _p(workspace), workspace.numel() * workspace.element_size(),
                                       _stream(stream)), "fastkv_decode_attn")
+
+
+def fastkv_prefill_workspace_bytes(shape: Shape) -> int:
+    n = ctypes.c_size_t(0)
+    _check(_load().fastkv_prefill_workspace_bytes(ctypes.byref(shape), ctypes.byref(n)), "fastkv_prefill_workspace_bytes")
+    return int(n.value)
+
+
+def fastkv_prefill_attention(shape: Shape, q, k, v, out, scores_kv, scores_tsp, workspace, stream=None) -> None:
+    _check(_load().fastkv_prefill_attention(ctypes.byref(shape), _p(q), _p(k), _p(v), _p(out), _p(scores_kv),
+                                            _p(scores_tsp), _p(workspace), workspace.numel() * workspace.element_size(),
+                                            _stream(stream)), "fastkv_prefill_attention")
 
 
 def fastkv_device_status(workspace, stream=None):

@@ -8,8 +8,8 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libfastkv_b200.so")
-SOURCES = ["api.cu", "score.cu", "score_fused.cu", "score_parked.cu", "select.cu", "compact.cu", "decode_attn.cu", "score_static.cu"]
-HEADERS = ["common.cuh", "score.cuh", "select.cuh", "compact.cuh", "decode_attn.cuh", os.path.join("..", "..", "include", "fastkv.h")]
+SOURCES = ["api.cu", "score.cu", "score_fused.cu", "score_parked.cu", "select.cu", "compact.cu", "decode_attn.cu", "score_static.cu", "prefill_attn.cu"]
+HEADERS = ["common.cuh", "score.cuh", "select.cuh", "compact.cuh", "decode_attn.cuh", "prefill_attn.cuh", os.path.join("..", "..", "include", "fastkv.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--shared"]
 

@@ -11,6 +11,7 @@
 
 #include "compact.cuh"
 #include "decode_attn.cuh"
+#include "prefill_attn.cuh"
 #include "score.cuh"
 #include "select.cuh"
 
@@ -48,8 +49,10 @@ struct DebugConfig {
 DebugConfig g_debug;
 
 // ---- optional per-kernel timing ("time_kernels" hook): a pair of events around every launch ----------
-enum KernelId { KID_SCORE = 0, KID_POOL = 1, KID_SELECT = 2, KID_COMPACT = 3, KID_DECODE = 4, KID_COUNT = 5 };
-const char* const kKernelNames[KID_COUNT] = {"score", "pool", "select", "compact", "decode_attn"};
+enum KernelId { KID_SCORE = 0, KID_POOL = 1, KID_SELECT = 2, KID_COMPACT = 3, KID_DECODE = 4, KID_PREFILL = 5,
+                KID_WINDOW_SCORES = 6, KID_COUNT = 7 };
+const char* const kKernelNames[KID_COUNT] = {"score", "pool", "select", "compact", "decode_attn", "prefill_attn",
+                                             "window_scores"};
 struct KernelTimes {
   bool on = false;
   std::mutex mu;
@@ -642,6 +645,119 @@ int fastkv_decode_attn(const fastkv_shape* shape, const void* q, const void* k_c
   }
   if (e != cudaSuccess) return cuda_fail(e, "decode_attn_kernel launch");
   g_launches += 2;
+  return FASTKV_OK;
+}
+
+// ---- prefill attention with the scores as a by-product ------------------------------------------------
+namespace {
+struct PrefillLayout {
+  size_t off_wstat, off_a, off_wlog, bytes;
+  long long ld;
+  int rows;                     // un-pooled rows the pooling kernel reads
+};
+PrefillLayout prefill_layout(const fastkv_shape& s) {
+  PrefillLayout l;
+  const bool per_head = s.agg_order == FASTKV_POOL_THEN_GROUP;
+  l.rows = per_head ? s.n_q_heads : s.n_kv_heads;
+  l.ld = static_cast<long long>(round_up(static_cast<size_t>(s.total_len), 64));
+  size_t off = sizeof(WorkspaceHeader);
+  l.off_wstat = off;
+  off += round_up(sizeof(float2) * static_cast<size_t>(s.batch) * s.n_q_heads * s.window, 256);
+  l.off_a = off;
+  off += round_up(sizeof(float) * static_cast<size_t>(l.rows) * l.ld, 256);
+  l.off_wlog = off;
+  off += round_up(sizeof(float) * static_cast<size_t>(s.n_q_heads) * s.window * l.ld, 256);
+  l.bytes = off;
+  return l;
+}
+int check_prefill_shape(const fastkv_shape* s) {
+  int rc = check_shape(s, true);
+  if (rc) return rc;
+  if (s->q_layout != FASTKV_Q_FULL) return fail(FASTKV_ERR_INVALID_ARG, "prefill attention needs the full packed Q (FASTKV_Q_FULL)");
+  if (s->v_stride_tok % 8 || s->v_stride_head % 8)
+    return fail(FASTKV_ERR_UNSUPPORTED, "v strides must be multiples of 8 elements (16 bytes)");
+  if (s->v_stride_head < s->head_dim || s->v_stride_tok < s->head_dim)
+    return fail(FASTKV_ERR_INVALID_ARG, "v strides are smaller than head_dim");
+  return FASTKV_OK;
+}
+}  // namespace
+
+int fastkv_prefill_workspace_bytes(const fastkv_shape* shape, size_t* bytes) {
+  int rc = check_prefill_shape(shape);
+  if (rc) return rc;
+  if (bytes == nullptr) return fail(FASTKV_ERR_INVALID_ARG, "bytes is NULL");
+  *bytes = prefill_layout(*shape).bytes;
+  return FASTKV_OK;
+}
+
+int fastkv_prefill_attention(const fastkv_shape* shape, const void* q, const void* k, const void* v, void* out,
+                             float* scores_kv, float* scores_tsp, void* workspace, size_t workspace_bytes,
+                             void* stream_) {
+  int rc = check_prefill_shape(shape);
+  if (rc) return rc;
+  if (!q || !k || !v || !out) return fail(FASTKV_ERR_INVALID_ARG, "prefill_attention: q, k, v and out are required");
+  if (scores_tsp != nullptr && scores_kv == nullptr)
+    return fail(FASTKV_ERR_INVALID_ARG, "prefill_attention: scores_tsp needs scores_kv");
+  if (reinterpret_cast<uintptr_t>(out) % 16) return fail(FASTKV_ERR_UNSUPPORTED, "prefill_attention: out must be 16-byte aligned");
+  const fastkv_shape& s = *shape;
+  const PrefillLayout lay = prefill_layout(s);
+  const bool want_scores = scores_kv != nullptr;
+  if ((rc = check_workspace(workspace, workspace_bytes, want_scores ? lay.bytes : sizeof(WorkspaceHeader)))) return rc;
+  if ((rc = check_device())) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int G = s.n_q_heads / s.n_kv_heads;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  CUtensorMap tmap_q, tmap_k, tmap_v;
+  if ((rc = encode_bf16_3d(&tmap_q, q, s.head_dim, s.n_q_heads, s.total_len, s.q_stride_head, s.q_stride_tok, 1, 128)) ||
+      (rc = encode_bf16_3d(&tmap_k, k, s.head_dim, s.n_kv_heads, s.total_len, s.k_stride_head, s.k_stride_tok, 1, 128)) ||
+      (rc = encode_bf16_3d(&tmap_v, v, s.head_dim, s.n_kv_heads, s.total_len, s.v_stride_head, s.v_stride_tok, 1, 128)))
+    return rc;
+  cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(WorkspaceHeader), stream);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace header)");
+  const float scale = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / std::sqrt(static_cast<float>(s.head_dim));
+  PrefillParams pp;
+  pp.batch = s.batch; pp.total_len = s.total_len; pp.n_q_heads = s.n_q_heads; pp.group = G; pp.window = s.window;
+  pp.scale_log2 = scale * 1.4426950408889634f;
+  pp.cu_seqlens = s.cu_seqlens;
+  pp.out = out;
+  pp.out_stride_tok = static_cast<long long>(s.n_q_heads) * s.head_dim;      // dense [total_len, n_q_heads, head_dim]
+  pp.out_stride_head = s.head_dim;
+  pp.wlog = want_scores ? reinterpret_cast<float*>(ws + lay.off_wlog) : nullptr;
+  pp.ld_w = lay.ld;
+  pp.wstat = reinterpret_cast<float2*>(ws + lay.off_wstat);
+  pp.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+  pp.wait_limit = g_debug.wait_limit_cycles > 0 ? g_debug.wait_limit_cycles : kWaitLimitCycles;
+  {
+    TimedLaunch timed(KID_PREFILL, stream);
+    e = launch_prefill_attn(s.head_dim, tmap_q, tmap_k, tmap_v, pp, s.max_len, stream);
+  }
+  if (e != cudaSuccess) return cuda_fail(e, "prefill_attn_kernel launch");
+  ++g_launches;
+  if (!want_scores) return FASTKV_OK;
+  WindowScoresParams wp;
+  wp.total_len = s.total_len; wp.n_q_heads = s.n_q_heads; wp.n_kv_heads = s.n_kv_heads; wp.group = G; wp.window = s.window;
+  wp.per_head = s.agg_order == FASTKV_POOL_THEN_GROUP;
+  wp.cu_seqlens = s.cu_seqlens; wp.wlog = pp.wlog; wp.ld_w = lay.ld; wp.wstat = pp.wstat;
+  wp.a_out = reinterpret_cast<float*>(ws + lay.off_a); wp.ld_a = lay.ld;
+  {
+    TimedLaunch timed(KID_WINDOW_SCORES, stream);
+    e = launch_window_scores(wp, s.max_len, s.batch, stream);
+  }
+  if (e != cudaSuccess) return cuda_fail(e, "window_scores_kernel launch");
+  ++g_launches;
+  PoolRowsParams rp;
+  rp.total_len = s.total_len; rp.n_kv_heads = s.n_kv_heads; rp.group = G; rp.window = s.window;
+  rp.per_head = wp.per_head; rp.pool_kernel = s.pool_kernel; rp.pool_mode = s.pool_mode;
+  rp.cu_seqlens = s.cu_seqlens; rp.a = wp.a_out; rp.ld_a = lay.ld;
+  rp.scores_kv = scores_kv; rp.ld_scores = s.total_len; rp.scores_tsp = scores_tsp;
+  if (sizeof(float) * static_cast<size_t>(lay.rows) * (kPoolKeys + s.pool_kernel) > 200 * 1024)
+    return fail(FASTKV_ERR_UNSUPPORTED, "heads x pool halo do not fit the pooling kernel's shared memory");
+  {
+    TimedLaunch timed(KID_POOL, stream);
+    e = launch_pool_rows(rp, s.max_len, s.batch, stream);
+  }
+  if (e != cudaSuccess) return cuda_fail(e, "pool_rows_kernel launch");
+  ++g_launches;
   return FASTKV_OK;
 }
 

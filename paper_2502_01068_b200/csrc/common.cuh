@@ -45,6 +45,16 @@ enum Site : int {
   SITE_PARKED_REF = 23,
   SITE_PARKED_STATS = 24,
   SITE_PARKED_NORM = 25,
+  SITE_ATTN_RING = 26,
+  SITE_ATTN_DRAIN = 27,
+  SITE_ATTN_Q = 28,
+  SITE_ATTN_K = 29,
+  SITE_ATTN_V = 30,
+  SITE_ATTN_P = 31,
+  SITE_ATTN_S = 32,
+  SITE_ATTN_SFULL = 33,
+  SITE_ATTN_PFREE = 34,
+  SITE_ATTN_ODONE = 35,
 };
 
 // Records `text` as the calling thread's last error (see fastkv_last_error) and returns `status`.

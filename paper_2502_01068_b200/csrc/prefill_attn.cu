@@ -1,0 +1,433 @@
+// Causal prefill attention of a whole prompt that hands out the saliency scores as a by-product
+// (Alg. 1: the TSP layer's own attention produces Att_l; Sec. 4.2 / App. D.4: the token importance
+// estimation is otherwise a separate pass over Q_window x K).
+//
+// One CTA per (128-query tile, query head); it walks the key tiles 0 .. tile of its last query:
+//
+//   producer   one thread: the Q tile once, then K and V tiles into two-stage rings by TMA;
+//   issuer     one thread: S = Q K^T (tcgen05.mma, 128 x 128 x d, fp32 in tensor memory, two S buffers so
+//              that the contraction of tile j+1 runs while tile j is in the softmax), then
+//              O += P V with P (bf16) from shared memory and V as an MN-major operand (the V tile is
+//              used as TMA delivers it, keys x d with d contiguous);
+//   softmax    four warps, one query row per thread (tensor-memory lane = row): online softmax in
+//              log2 units with a lazily raised reference (the row's reference moves, and its O row is
+//              rescaled, only when a logit exceeds it by more than 8 binary orders of magnitude),
+//              P rounded to bf16 into the 128-byte-swizzled K-major layout the second contraction
+//              reads, and at the end O / l -> bf16 -> global memory.
+//
+// The by-product: the threads whose query row is one of the last w of its sequence (the observation
+// window) also store their scaled logits of every key (fp32, log2 units) and, at the end, their
+// (reference, sum); window_scores_kernel turns these into Eq. 1's inner term summed over the window
+// and the GQA group, in the layout the pooling kernel of the scoring path reads.  No second pass over
+// K: what is added to the attention is w fp32 rows per query head.
+//
+// Every wait is bounded; a wait that gives up raises the status word and the CTA-wide abort flag, the
+// roles stop issuing work, copies and contractions in flight are waited for, tensor memory is released.
+#include "prefill_attn.cuh"
+
+namespace fastkv {
+
+namespace {
+
+constexpr int kBM = 128;                       // queries per CTA
+constexpr int kBN = 128;                       // keys per tile
+constexpr int kAttnThreads = 192;              // producer warp, issuer warp, four softmax warps
+constexpr int kChunkBytes = 128 * 128;         // 128 rows x 64 bf16: one swizzled column chunk of a tile
+constexpr float kRescaleSlackLog2 = 8.0f;
+
+template <int D>
+struct AttnCfg {
+  static constexpr int KH = D / 64;
+  static constexpr int kTileBytes = KH * kChunkBytes;     // Q, K or V tile
+  static constexpr int kPBytes = 2 * kChunkBytes;         // P: 128 queries x 128 keys bf16
+  static constexpr int kSmemBytes = 1024 + 5 * kTileBytes + kPBytes + 256;
+};
+
+struct AttnBarriers {
+  uint64_t q_full;
+  uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
+  uint64_t s_full[2], s_free[2];
+  uint64_t p_full, p_free;
+  uint64_t o_done;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+// MN-major operand tile as TMA writes it (rows of 128 bytes = 64 elements of the MN dimension, one row per
+// K index, 128-byte swizzle): 64-element MN chunks are `chunk_bytes` apart (leading byte offset), groups of
+// eight K rows 1024 bytes apart (stride byte offset).
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint32_t chunk_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>((chunk_bytes >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+}  // namespace
+
+template <int D>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                    const __grid_constant__ CUtensorMap tmap_v, const PrefillParams p) {
+  using Cfg = AttnCfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  uint8_t* sQ = smem;
+  uint8_t* sK = sQ + Cfg::kTileBytes;                     // two stages
+  uint8_t* sV = sK + 2 * Cfg::kTileBytes;                 // two stages
+  uint8_t* sP = sV + 2 * Cfg::kTileBytes;
+  AttnBarriers* bars = reinterpret_cast<AttnBarriers*>(sP + Cfg::kPBytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.z, h = blockIdx.y, g = h / p.group;
+  const int row0 = p.cu_seqlens ? p.cu_seqlens[b] : 0;
+  const int L = p.cu_seqlens ? p.cu_seqlens[b + 1] - row0 : p.total_len;
+  const int n_qtiles = (L + kBM - 1) / kBM;
+  const int qi = n_qtiles - 1 - static_cast<int>(blockIdx.x);      // the longest rows first
+  if (qi < 0) return;                                              // (uniform per CTA, before any barrier)
+  const int q0 = qi * kBM;
+  const int n_tiles = qi + 1;                                      // key tiles 0 .. qi (causal)
+  const long long limit = p.wait_limit;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&bars->q_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], 1);
+      mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], 1);
+      mbar_init(&bars->s_full[i], 1); mbar_init(&bars->s_free[i], 4);
+    }
+    mbar_init(&bars->p_full, 4);
+    mbar_init(&bars->p_free, 1);
+    mbar_init(&bars->o_done, 1);
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    tma_prefetch_desc(&tmap_q);
+    tma_prefetch_desc(&tmap_k);
+    tma_prefetch_desc(&tmap_v);
+  }
+  if (warp == 1) {
+    tmem_alloc(&bars->tmem_base, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = bars->tmem_base;
+  volatile int* abort_flag = &bars->abort_flag;
+  pdl_launch_dependents();
+  pdl_wait();
+
+  if (warp == 0) {
+    // ---------------- producer ----------------
+    if (lane == 0) {
+      const uint64_t pol_q = l2_policy_evict_first();      // a Q tile is read by one CTA
+      const uint64_t pol_kv = l2_policy_evict_last();      // K / V tiles are read by every later query tile
+      mbar_arrive_expect_tx(&bars->q_full, Cfg::kTileBytes);
+      for (int c = 0; c < Cfg::KH; ++c) tma_load_3d(sQ + c * kChunkBytes, &tmap_q, &bars->q_full, c * 64, h, row0 + q0, pol_q);
+      bool ok = true;
+      int issued = 0;
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int s = j & 1;
+        ok = mbar_wait_bounded(&bars->k_empty[s], ((j >> 1) & 1) ^ 1, abort_flag, p.hdr, SITE_ATTN_RING, limit);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&bars->k_full[s], Cfg::kTileBytes);
+        for (int c = 0; c < Cfg::KH; ++c)
+          tma_load_3d(sK + s * Cfg::kTileBytes + c * kChunkBytes, &tmap_k, &bars->k_full[s], c * 64, g, row0 + j * kBN, pol_kv);
+        ok = mbar_wait_bounded(&bars->v_empty[s], ((j >> 1) & 1) ^ 1, abort_flag, p.hdr, SITE_ATTN_RING, limit);
+        if (!ok) {                                          // K of this tile is in flight, V is not
+          mbar_wait_drain(&bars->k_full[s], (j >> 1) & 1, p.hdr, SITE_ATTN_DRAIN, limit);
+          break;
+        }
+        mbar_arrive_expect_tx(&bars->v_full[s], Cfg::kTileBytes);
+        for (int c = 0; c < Cfg::KH; ++c)
+          tma_load_3d(sV + s * Cfg::kTileBytes + c * kChunkBytes, &tmap_v, &bars->v_full[s], c * 64, g, row0 + j * kBN, pol_kv);
+        issued = j + 1;
+      }
+      // nothing may still be landing in shared memory when the CTA ends
+      mbar_wait_drain(&bars->q_full, 0, p.hdr, SITE_ATTN_DRAIN, limit);
+      for (int j = max(0, issued - 2); j < issued; ++j) {
+        mbar_wait_drain(&bars->k_full[j & 1], (j >> 1) & 1, p.hdr, SITE_ATTN_DRAIN, limit);
+        mbar_wait_drain(&bars->v_full[j & 1], (j >> 1) & 1, p.hdr, SITE_ATTN_DRAIN, limit);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = umma_idesc_bf16_f32(kBM, kBN);
+      constexpr uint32_t idesc_o = umma_idesc_bf16_f32(kBM, D) | (1u << 16);      // B (V) is MN-major
+      const uint32_t q_addr = smem_u32(sQ), p_addr = smem_u32(sP);
+      bool ok = mbar_wait_bounded(&bars->q_full, 0, abort_flag, p.hdr, SITE_ATTN_Q, limit);
+      int committed = 0;
+      auto second = [&](int t) {                           // O (+)= P_t V_t
+        const int s = t & 1;
+        ok = mbar_wait_bounded(&bars->v_full[s], (t >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit) &&
+             mbar_wait_bounded(&bars->p_full, t & 1, abort_flag, p.hdr, SITE_ATTN_P, limit);
+        if (!ok) return;
+        tc_fence_after_sync();
+        const uint32_t v_addr = smem_u32(sV + s * Cfg::kTileBytes);
+#pragma unroll
+        for (int kk = 0; kk < kBN / 16; ++kk) {
+          const uint64_t adesc = umma_desc_k_sw128(p_addr + (kk >> 2) * kChunkBytes + (kk & 3) * 32);
+          const uint64_t bdesc = umma_desc_mn_sw128(v_addr + kk * 2048, kChunkBytes);
+          tc_mma_bf16(tmem_base + 256, adesc, bdesc, idesc_o, (t > 0 || kk > 0) ? 1u : 0u);
+        }
+        tc_commit(&bars->v_empty[s]);
+        tc_commit(&bars->p_free);
+        ++committed;
+      };
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int s = j & 1;
+        ok = mbar_wait_bounded(&bars->k_full[s], (j >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit) &&
+             mbar_wait_bounded(&bars->s_free[s], ((j >> 1) & 1) ^ 1, abort_flag, p.hdr, SITE_ATTN_S, limit);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t k_addr = smem_u32(sK + s * Cfg::kTileBytes);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint64_t adesc = umma_desc_k_sw128(q_addr + (kk >> 2) * kChunkBytes + (kk & 3) * 32);
+          const uint64_t bdesc = umma_desc_k_sw128(k_addr + (kk >> 2) * kChunkBytes + (kk & 3) * 32);
+          tc_mma_bf16(tmem_base + s * kBN, adesc, bdesc, idesc_s, kk > 0 ? 1u : 0u);
+        }
+        tc_commit(&bars->k_empty[s]);
+        tc_commit(&bars->s_full[s]);
+        ++committed;
+        if (j >= 1) second(j - 1);
+      }
+      if (ok) second(n_tiles - 1);
+      // every contraction issued has finished before tensor memory is released (and O is complete)
+      if (committed > 0) {
+        tc_commit(&bars->o_done);
+        mbar_wait_drain(&bars->o_done, 0, p.hdr, SITE_ATTN_DRAIN, limit);
+      }
+    }
+  } else {
+    // ---------------- softmax: one query row per thread ----------------
+    const int quarter = warp & 3;
+    const int r = quarter * 32 + lane;                    // row of the tile = tensor-memory lane
+    const int t = q0 + r;                                 // query position in its sequence
+    const int t_eff = min(t, L - 1);                      // rows past the end repeat the last row (never stored)
+    const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    const int jw = t - (L - p.window);                    // window row index, if 0 <= jw < w
+    const bool is_window = p.wlog != nullptr && jw >= 0 && t < L;
+    float* const wlog_row = is_window ? p.wlog + (static_cast<size_t>(h) * p.window + jw) * p.ld_w + row0 : nullptr;
+    float m_ref = -INFINITY, l = 0.0f;
+    bool ok = true;
+    for (int j = 0; j < n_tiles; ++j) {
+      const int s = j & 1;
+      if (ok) ok = mbar_wait_bounded(&bars->s_full[s], (j >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_SFULL, limit);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const int key0 = j * kBN;
+      const bool diagonal = key0 + kBN - 1 > t_eff;       // some keys of the tile are not visible to this row
+      // first reading of the row: its largest visible logit
+      float tile_max = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < kBN / 32; ++c) {
+        float v[32];
+        tmem_ld_32x32(lane_addr + s * kBN + c * 32, v);
+        if (diagonal) {
+#pragma unroll
+          for (int x = 0; x < 32; ++x) tile_max = fmaxf(tile_max, key0 + c * 32 + x <= t_eff ? v[x] : -INFINITY);
+        } else {
+#pragma unroll
+          for (int x = 0; x < 32; ++x) tile_max = fmaxf(tile_max, v[x]);
+        }
+      }
+      tile_max *= p.scale_log2;                            // the scale is positive
+      // the reference moves only when the tile's maximum is far above it (or at the first tile)
+      const bool move = tile_max > m_ref + kRescaleSlackLog2;
+      const float alpha = move ? ex2(m_ref - tile_max) : 1.0f;     // 0 at the first tile
+      if (move) { m_ref = tile_max; l *= alpha; }
+      // P of the previous tile has been consumed (so has O been updated) before O is rescaled and P rewritten
+      if (j >= 1) {
+        if (ok) ok = mbar_wait_bounded(&bars->p_free, (j - 1) & 1, abort_flag, p.hdr, SITE_ATTN_PFREE, limit);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+        if (__any_sync(0xffffffffu, move)) {
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            float o[32];
+            tmem_ld_32x32(lane_addr + 256 + c * 32, o);
+#pragma unroll
+            for (int x = 0; x < 32; ++x) o[x] *= alpha;
+            tmem_st_32x32(lane_addr + 256 + c * 32, o);
+          }
+          tmem_wait_st();
+        }
+      }
+      // second reading: p = exp2(s - ref), the row sum, P in bf16 for the second contraction
+      float lsum = 0.0f;
+#pragma unroll
+      for (int c = 0; c < kBN / 32; ++c) {
+        float v[32];
+        tmem_ld_32x32(lane_addr + s * kBN + c * 32, v);
+        if (c == kBN / 32 - 1) {                           // the S buffer is in registers: the issuer may overwrite it
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars->s_free[s]);
+        }
+#pragma unroll
+        for (int x = 0; x < 32; ++x) {
+          const float sl = v[x] * p.scale_log2;
+          const bool vis = !diagonal || key0 + c * 32 + x <= t_eff;
+          v[x] = vis ? sl : -INFINITY;
+        }
+        if (is_window) {                                   // by-product: this row's logits (log2 units), masked = -inf
+#pragma unroll
+          for (int x = 0; x < 32; ++x)
+            if (key0 + c * 32 + x < L) wlog_row[key0 + c * 32 + x] = v[x];
+        }
+#pragma unroll
+        for (int x = 0; x < 32; ++x) {
+          v[x] = ex2(v[x] - m_ref);
+          lsum += v[x];
+        }
+        // 8 keys = 16 bytes per store; 16-byte unit u of row r sits at unit (u ^ (r & 7)) of the row's 128 bytes
+        uint8_t* const prow = sP + (c >> 1) * kChunkBytes + r * 128;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int unit = (c & 1) * 4 + u;
+          uint4 w4;
+          w4.x = pack_bf16(v[u * 8 + 0], v[u * 8 + 1]);
+          w4.y = pack_bf16(v[u * 8 + 2], v[u * 8 + 3]);
+          w4.z = pack_bf16(v[u * 8 + 4], v[u * 8 + 5]);
+          w4.w = pack_bf16(v[u * 8 + 6], v[u * 8 + 7]);
+          *reinterpret_cast<uint4*>(prow + ((unit ^ (r & 7)) << 4)) = w4;
+        }
+      }
+      l += lsum;
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core's proxy
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->p_full);
+    }
+    // the finished row: O / l -> bf16
+    if (ok) ok = mbar_wait_bounded(&bars->o_done, 0, abort_flag, p.hdr, SITE_ATTN_ODONE, limit);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after_sync();
+      const float inv_l = 1.0f / l;
+      uint8_t* const orow = reinterpret_cast<uint8_t*>(p.out) +
+                            (static_cast<size_t>(row0 + t) * p.out_stride_tok + static_cast<size_t>(h) * p.out_stride_head) * 2;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        float o[32];
+        tmem_ld_32x32(lane_addr + 256 + c * 32, o);
+        if (t < L) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            uint4 w4;
+            w4.x = pack_bf16(o[u * 8 + 0] * inv_l, o[u * 8 + 1] * inv_l);
+            w4.y = pack_bf16(o[u * 8 + 2] * inv_l, o[u * 8 + 3] * inv_l);
+            w4.z = pack_bf16(o[u * 8 + 4] * inv_l, o[u * 8 + 5] * inv_l);
+            w4.w = pack_bf16(o[u * 8 + 6] * inv_l, o[u * 8 + 7] * inv_l);
+            *reinterpret_cast<uint4*>(orow + c * 64 + u * 16) = w4;
+          }
+        }
+      }
+      if (is_window) p.wstat[(static_cast<size_t>(b) * p.n_q_heads + h) * p.window + jw] = make_float2(m_ref, l);
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Eq. 1's inner term from the window rows' logits: for key i of KV head g,
+//   a[g, i] = sum over the query heads h of the group and the window rows j with i <= L - w + j of
+//             exp2(s[h, j, i] - ref[h, j]) / l[h, j]
+// (one row per query head instead with per_head).  One thread per key.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) window_scores_kernel(const WindowScoresParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int b = blockIdx.y;
+  const int row0 = p.cu_seqlens ? p.cu_seqlens[b] : 0;
+  const int L = p.cu_seqlens ? p.cu_seqlens[b + 1] - row0 : p.total_len;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= L || L < p.window) return;
+  const int G = p.group, w = p.window;
+  for (int g = 0; g < p.n_kv_heads; ++g) {
+    float a_g = 0.0f;
+    for (int hl = 0; hl < G; ++hl) {
+      const int h = g * G + hl;
+      float a_h = 0.0f;
+      for (int j = 0; j < w; ++j) {
+        if (i > L - w + j) continue;                       // causal: key i is not visible to window row j
+        const float2 st = p.wstat[(static_cast<size_t>(b) * p.n_q_heads + h) * w + j];
+        const float s = p.wlog[(static_cast<size_t>(h) * w + j) * p.ld_w + row0 + i];
+        a_h += ex2(s - st.x) / st.y;
+      }
+      if (p.per_head) p.a_out[static_cast<size_t>(h) * p.ld_a + row0 + i] = a_h;
+      a_g += a_h;
+    }
+    if (!p.per_head) p.a_out[static_cast<size_t>(g) * p.ld_a + row0 + i] = a_g;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+
+template <int D>
+static cudaError_t launch_attn_t(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                                 const PrefillParams& p, int max_len, cudaStream_t stream) {
+  using Cfg = AttnCfg<D>;
+  static PerDeviceOnce configured;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (!configured.done(dev)) {
+    e = cudaFuncSetAttribute(prefill_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured.set(dev);
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((max_len + kBM - 1) / kBM, p.n_q_heads, p.batch);
+  cfg.blockDim = dim3(kAttnThreads);
+  cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  fill_pdl_attribute(&attr[0]);
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, prefill_attn_kernel<D>, tq, tk, tv, p);
+}
+
+cudaError_t launch_prefill_attn(int head_dim, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                                const PrefillParams& p, int max_len, cudaStream_t stream) {
+  if (head_dim == 128) return launch_attn_t<128>(tq, tk, tv, p, max_len, stream);
+  if (head_dim == 64) return launch_attn_t<64>(tq, tk, tv, p, max_len, stream);
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_window_scores(const WindowScoresParams& p, int max_len, int batch, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((max_len + 255) / 256, batch);
+  cfg.blockDim = dim3(256);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  fill_pdl_attribute(&attr[0]);
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, window_scores_kernel, p);
+}
+
+}  // namespace fastkv
