@@ -40,14 +40,14 @@ struct AttnCfg {
   static constexpr int KH = D / 64;
   static constexpr int kTileBytes = KH * kChunkBytes;     // Q, K or V tile
   static constexpr int kPBytes = 2 * kChunkBytes;         // P: 128 queries x 128 keys bf16
-  static constexpr int kSmemBytes = 1024 + 5 * kTileBytes + kPBytes + 256;
+  static constexpr int kSmemBytes = 1024 + 5 * kTileBytes + 2 * kPBytes + 256;
 };
 
 struct AttnBarriers {
   uint64_t q_full;
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
   uint64_t s_full[2], s_free[2];
-  uint64_t p_full, p_free;
+  uint64_t p_full[2], p_free[2];
   uint64_t o_done;
   uint32_t tmem_base;
   int abort_flag;
@@ -85,7 +85,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   uint8_t* sK = sQ + Cfg::kTileBytes;                     // two stages
   uint8_t* sV = sK + 2 * Cfg::kTileBytes;                 // two stages
   uint8_t* sP = sV + 2 * Cfg::kTileBytes;
-  AttnBarriers* bars = reinterpret_cast<AttnBarriers*>(sP + Cfg::kPBytes);
+  AttnBarriers* bars = reinterpret_cast<AttnBarriers*>(sP + 2 * Cfg::kPBytes);   // P is double-buffered
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.z, h = blockIdx.y, g = h / p.group;
@@ -105,8 +105,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], 1);
       mbar_init(&bars->s_full[i], 1); mbar_init(&bars->s_free[i], 4);
     }
-    mbar_init(&bars->p_full, 4);
-    mbar_init(&bars->p_free, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&bars->p_full[i], 4); mbar_init(&bars->p_free[i], 1); }
     mbar_init(&bars->o_done, 1);
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -171,18 +170,18 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       auto second = [&](int t) {                           // O (+)= P_t V_t
         const int s = t & 1;
         ok = mbar_wait_bounded(&bars->v_full[s], (t >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit) &&
-             mbar_wait_bounded(&bars->p_full, t & 1, abort_flag, p.hdr, SITE_ATTN_P, limit);
+             mbar_wait_bounded(&bars->p_full[s], (t >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_P, limit);
         if (!ok) return;
         tc_fence_after_sync();
         const uint32_t v_addr = smem_u32(sV + s * Cfg::kTileBytes);
 #pragma unroll
         for (int kk = 0; kk < kBN / 16; ++kk) {
-          const uint64_t adesc = umma_desc_k_sw128(p_addr + (kk >> 2) * kChunkBytes + (kk & 3) * 32);
+          const uint64_t adesc = umma_desc_k_sw128(p_addr + s * Cfg::kPBytes + (kk >> 2) * kChunkBytes + (kk & 3) * 32);
           const uint64_t bdesc = umma_desc_mn_sw128(v_addr + kk * 2048, kChunkBytes);
           tc_mma_bf16(tmem_base + 256, adesc, bdesc, idesc_o, (t > 0 || kk > 0) ? 1u : 0u);
         }
         tc_commit(&bars->v_empty[s]);
-        tc_commit(&bars->p_free);
+        tc_commit(&bars->p_free[s]);
         ++committed;
       };
       for (int j = 0; j < n_tiles && ok; ++j) {
@@ -230,88 +229,87 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       tc_fence_after_sync();
       const int key0 = j * kBN;
       const bool diagonal = key0 + kBN - 1 > t_eff;       // some keys of the tile are not visible to this row
-      // first reading of the row: its largest visible logit
-      float tile_max = -INFINITY;
+      // the whole row of the tile in registers; the S buffer goes back to the issuer at once
+      float v[kBN];
 #pragma unroll
-      for (int c = 0; c < kBN / 32; ++c) {
-        float v[32];
-        tmem_ld_32x32(lane_addr + s * kBN + c * 32, v);
-        if (diagonal) {
+      for (int c = 0; c < kBN / 32; ++c) tmem_ld_32x32(lane_addr + s * kBN + c * 32, *reinterpret_cast<float (*)[32]>(&v[c * 32]));
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->s_free[s]);
+      if (diagonal) {
 #pragma unroll
-          for (int x = 0; x < 32; ++x) tile_max = fmaxf(tile_max, key0 + c * 32 + x <= t_eff ? v[x] : -INFINITY);
-        } else {
-#pragma unroll
-          for (int x = 0; x < 32; ++x) tile_max = fmaxf(tile_max, v[x]);
-        }
+        for (int x = 0; x < kBN; ++x) v[x] = key0 + x <= t_eff ? v[x] : -INFINITY;
       }
-      tile_max *= p.scale_log2;                            // the scale is positive
+      float mx[4] = {v[0], v[1], v[2], v[3]};
+#pragma unroll
+      for (int x = 4; x < kBN; x += 4) {
+        mx[0] = fmaxf(mx[0], v[x]); mx[1] = fmaxf(mx[1], v[x + 1]); mx[2] = fmaxf(mx[2], v[x + 2]); mx[3] = fmaxf(mx[3], v[x + 3]);
+      }
+      const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;   // the scale is positive
       // the reference moves only when the tile's maximum is far above it (or at the first tile)
       const bool move = tile_max > m_ref + kRescaleSlackLog2;
       const float alpha = move ? ex2(m_ref - tile_max) : 1.0f;     // 0 at the first tile
       if (move) { m_ref = tile_max; l *= alpha; }
-      // P of the previous tile has been consumed (so has O been updated) before O is rescaled and P rewritten
-      if (j >= 1) {
-        if (ok) ok = mbar_wait_bounded(&bars->p_free, (j - 1) & 1, abort_flag, p.hdr, SITE_ATTN_PFREE, limit);
+      if (j >= 1 && __any_sync(0xffffffffu, move)) {
+        // O is rescaled once the second contraction of the tile before has been added to it
+        if (ok) ok = mbar_wait_bounded(&bars->p_free[(j - 1) & 1], ((j - 1) >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_PFREE, limit);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after_sync();
-        if (__any_sync(0xffffffffu, move)) {
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            float o[32];
-            tmem_ld_32x32(lane_addr + 256 + c * 32, o);
+        for (int c = 0; c < D / 32; ++c) {
+          float o[32];
+          tmem_ld_32x32(lane_addr + 256 + c * 32, o);
 #pragma unroll
-            for (int x = 0; x < 32; ++x) o[x] *= alpha;
-            tmem_st_32x32(lane_addr + 256 + c * 32, o);
-          }
-          tmem_wait_st();
+          for (int x = 0; x < 32; ++x) o[x] *= alpha;
+          tmem_st_32x32(lane_addr + 256 + c * 32, o);
+        }
+        tmem_wait_st();
+      }
+      if (is_window) {                                     // by-product: this row's logits (log2 units), masked = -inf
+        float* const dst = wlog_row + key0;
+        if (key0 + kBN <= L && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+#pragma unroll
+          for (int x = 0; x < kBN; x += 4)
+            *reinterpret_cast<float4*>(dst + x) = make_float4(v[x] * p.scale_log2, v[x + 1] * p.scale_log2,
+                                                              v[x + 2] * p.scale_log2, v[x + 3] * p.scale_log2);
+        } else {
+#pragma unroll
+          for (int x = 0; x < kBN; ++x)
+            if (key0 + x < L) dst[x] = v[x] * p.scale_log2;
         }
       }
-      // second reading: p = exp2(s - ref), the row sum, P in bf16 for the second contraction
-      float lsum = 0.0f;
-#pragma unroll
-      for (int c = 0; c < kBN / 32; ++c) {
-        float v[32];
-        tmem_ld_32x32(lane_addr + s * kBN + c * 32, v);
-        if (c == kBN / 32 - 1) {                           // the S buffer is in registers: the issuer may overwrite it
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&bars->s_free[s]);
-        }
-#pragma unroll
-        for (int x = 0; x < 32; ++x) {
-          const float sl = v[x] * p.scale_log2;
-          const bool vis = !diagonal || key0 + c * 32 + x <= t_eff;
-          v[x] = vis ? sl : -INFINITY;
-        }
-        if (is_window) {                                   // by-product: this row's logits (log2 units), masked = -inf
-#pragma unroll
-          for (int x = 0; x < 32; ++x)
-            if (key0 + c * 32 + x < L) wlog_row[key0 + c * 32 + x] = v[x];
-        }
-#pragma unroll
-        for (int x = 0; x < 32; ++x) {
-          v[x] = ex2(v[x] - m_ref);
-          lsum += v[x];
-        }
-        // 8 keys = 16 bytes per store; 16-byte unit u of row r sits at unit (u ^ (r & 7)) of the row's 128 bytes
-        uint8_t* const prow = sP + (c >> 1) * kChunkBytes + r * 128;
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int unit = (c & 1) * 4 + u;
-          uint4 w4;
-          w4.x = pack_bf16(v[u * 8 + 0], v[u * 8 + 1]);
-          w4.y = pack_bf16(v[u * 8 + 2], v[u * 8 + 3]);
-          w4.z = pack_bf16(v[u * 8 + 4], v[u * 8 + 5]);
-          w4.w = pack_bf16(v[u * 8 + 6], v[u * 8 + 7]);
-          *reinterpret_cast<uint4*>(prow + ((unit ^ (r & 7)) << 4)) = w4;
-        }
+      // this P buffer was last read by the second contraction of tile j - 2
+      if (j >= 2) {
+        if (ok) ok = mbar_wait_bounded(&bars->p_free[s], ((j - 2) >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_PFREE, limit);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
       }
-      l += lsum;
+      // p = exp2(s * scale - ref), the row sum, P in bf16 for the second contraction
+      const float neg_ref = -m_ref;
+      float ls[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+      uint8_t* const pbuf = sP + s * Cfg::kPBytes + r * 128;
+#pragma unroll
+      for (int u = 0; u < kBN / 8; ++u) {                  // 8 keys = 16 bytes per store
+        float e[8];
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+          e[x] = ex2(fmaf(v[u * 8 + x], p.scale_log2, neg_ref));      // exp2(-inf) = 0 for a masked key
+          ls[x & 3] += e[x];
+        }
+        uint4 w4;
+        w4.x = pack_bf16(e[0], e[1]);
+        w4.y = pack_bf16(e[2], e[3]);
+        w4.z = pack_bf16(e[4], e[5]);
+        w4.w = pack_bf16(e[6], e[7]);
+        // 16-byte unit (u & 7) of row r sits at unit ((u & 7) ^ (r & 7)) of the row's 128 bytes in its 64-key chunk
+        *reinterpret_cast<uint4*>(pbuf + (u >> 3) * kChunkBytes + (((u & 7) ^ (r & 7)) << 4)) = w4;
+      }
+      l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core's proxy
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->p_full);
+      if (lane == 0) mbar_arrive(&bars->p_full[s]);
     }
     // the finished row: O / l -> bf16
     if (ok) ok = mbar_wait_bounded(&bars->o_done, 0, abort_flag, p.hdr, SITE_ATTN_ODONE, limit);
@@ -353,33 +351,39 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
 // Eq. 1's inner term from the window rows' logits: for key i of KV head g,
 //   a[g, i] = sum over the query heads h of the group and the window rows j with i <= L - w + j of
 //             exp2(s[h, j, i] - ref[h, j]) / l[h, j]
-// (one row per query head instead with per_head).  One thread per key.
+// (one row per query head instead with per_head).  One thread per key and KV head; G * w <= 64.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) window_scores_kernel(const WindowScoresParams p) {
+  __shared__ float2 st[64];                                // (reference, 1 / sum) of the group's G * w window rows
   pdl_launch_dependents();
   pdl_wait();
-  const int b = blockIdx.y;
+  const int b = blockIdx.z, g = blockIdx.y;
   const int row0 = p.cu_seqlens ? p.cu_seqlens[b] : 0;
   const int L = p.cu_seqlens ? p.cu_seqlens[b + 1] - row0 : p.total_len;
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= L || L < p.window) return;
+  if (L < p.window) return;
   const int G = p.group, w = p.window;
-  for (int g = 0; g < p.n_kv_heads; ++g) {
-    float a_g = 0.0f;
-    for (int hl = 0; hl < G; ++hl) {
-      const int h = g * G + hl;
-      float a_h = 0.0f;
-      for (int j = 0; j < w; ++j) {
-        if (i > L - w + j) continue;                       // causal: key i is not visible to window row j
-        const float2 st = p.wstat[(static_cast<size_t>(b) * p.n_q_heads + h) * w + j];
-        const float s = p.wlog[(static_cast<size_t>(h) * w + j) * p.ld_w + row0 + i];
-        a_h += ex2(s - st.x) / st.y;
-      }
-      if (p.per_head) p.a_out[static_cast<size_t>(h) * p.ld_a + row0 + i] = a_h;
-      a_g += a_h;
-    }
-    if (!p.per_head) p.a_out[static_cast<size_t>(g) * p.ld_a + row0 + i] = a_g;
+  if (threadIdx.x < G * w) {
+    const float2 v = p.wstat[(static_cast<size_t>(b) * p.n_q_heads + g * G) * w + threadIdx.x];
+    st[threadIdx.x] = make_float2(v.x, 1.0f / v.y);
   }
+  __syncthreads();
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= L) return;
+  const int first_j = max(0, i - (L - w));                 // causal: key i is visible to window rows j >= i - (L - w)
+  float a_g = 0.0f;
+  for (int hl = 0; hl < G; ++hl) {
+    const float* src = p.wlog + (static_cast<size_t>(g * G + hl) * w) * p.ld_w + row0 + i;
+    float a_h = 0.0f;
+#pragma unroll 8
+    for (int j = 0; j < w; ++j) {
+      const float s = j >= first_j ? __ldg(src + static_cast<size_t>(j) * p.ld_w) : -INFINITY;
+      const float2 rf = st[hl * w + j];
+      a_h += ex2(s - rf.x) * rf.y;
+    }
+    if (p.per_head) p.a_out[static_cast<size_t>(g * G + hl) * p.ld_a + row0 + i] = a_h;
+    a_g += a_h;
+  }
+  if (!p.per_head) p.a_out[static_cast<size_t>(g) * p.ld_a + row0 + i] = a_g;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -420,7 +424,7 @@ cudaError_t launch_prefill_attn(int head_dim, const CUtensorMap& tq, const CUten
 
 cudaError_t launch_window_scores(const WindowScoresParams& p, int max_len, int batch, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((max_len + 255) / 256, batch);
+  cfg.gridDim = dim3((max_len + 255) / 256, p.n_kv_heads, batch);
   cfg.blockDim = dim3(256);
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
