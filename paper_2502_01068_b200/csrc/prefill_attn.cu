@@ -7,13 +7,19 @@
 //   producer   one thread: the Q tile once, then K and V tiles into two-stage rings by TMA;
 //   issuer     one thread: S = Q K^T (tcgen05.mma, 128 x 128 x d, fp32 in tensor memory, two S buffers so
 //              that the contraction of tile j+1 runs while tile j is in the softmax), then
-//              O += P V with P (bf16) from shared memory and V as an MN-major operand (the V tile is
-//              used as TMA delivers it, keys x d with d contiguous);
-//   softmax    four warps, one query row per thread (tensor-memory lane = row): online softmax in
-//              log2 units with a lazily raised reference (the row's reference moves, and its O row is
-//              rescaled, only when a logit exceeds it by more than 8 binary orders of magnitude),
-//              P rounded to bf16 into the 128-byte-swizzled K-major layout the second contraction
-//              reads, and at the end O / l -> bf16 -> global memory.
+//              O += P V with P (bf16, packed two keys per column) read from tensor memory and V as an
+//              MN-major operand from shared memory (the V tile is used as TMA delivers it, keys x d
+//              with d contiguous).  With 128 x 128 tiles both operands of a contraction in shared
+//              memory would need all of its bandwidth (8 KB per 64 cycles), and K / V arrive and P would
+//              be written there as well: keeping P in tensor memory is what lets the tensor pipe run;
+//   softmax    eight warps, two threads per query row (tensor-memory lane = row; the two warps that
+//              share a lane quarter take 64 keys of the tile each and exchange their maxima through
+//              shared memory at one named barrier per tile): online softmax in log2 units with a
+//              lazily raised reference (the row's reference moves, and its O row is rescaled, only
+//              when a logit exceeds it by more than 8 binary orders of magnitude), P rounded to bf16
+//              and stored to tensor memory (two buffers), and at the end O / l -> bf16 -> global memory.
+//
+// Tensor memory (512 columns): S buffers at 0 and 128, O at 256, P buffers (64 columns each) at 384 and 448.
 //
 // The by-product: the threads whose query row is one of the last w of its sequence (the observation
 // window) also store their scaled logits of every key (fp32, log2 units) and, at the end, their
@@ -31,7 +37,8 @@ namespace {
 
 constexpr int kBM = 128;                       // queries per CTA
 constexpr int kBN = 128;                       // keys per tile
-constexpr int kAttnThreads = 192;              // producer warp, issuer warp, four softmax warps
+constexpr int kAttnThreads = 320;              // producer warp, issuer warp, eight softmax warps
+constexpr int kSoftmaxWarps = 8;
 constexpr int kChunkBytes = 128 * 128;         // 128 rows x 64 bf16: one swizzled column chunk of a tile
 constexpr float kRescaleSlackLog2 = 8.0f;
 
@@ -39,13 +46,13 @@ template <int D>
 struct AttnCfg {
   static constexpr int KH = D / 64;
   static constexpr int kTileBytes = KH * kChunkBytes;     // Q, K or V tile
-  static constexpr int kPBytes = 2 * kChunkBytes;         // P: 128 queries x 128 keys bf16
-  static constexpr int kSmemBytes = 1024 + 5 * kTileBytes + 2 * kPBytes + 256;
+  static constexpr int kKvStages = 3;
+  static constexpr int kSmemBytes = (1 + 2 * kKvStages) * kTileBytes + 256 + 2 * 2 * kBM * 4;
 };
 
 struct AttnBarriers {
   uint64_t q_full;
-  uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
+  uint64_t k_full[3], k_empty[3], v_full[3], v_empty[3];
   uint64_t s_full[2], s_free[2];
   uint64_t p_full[2], p_free[2];
   uint64_t o_done;
@@ -66,6 +73,17 @@ __device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint3
   return d;
 }
 
+// D[tmem] (+)= A[tmem] * B[smem]: A is read from tensor memory (lane = row, two bf16 per 32-bit column)
+__device__ __forceinline__ void tc_mma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -79,13 +97,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                     const __grid_constant__ CUtensorMap tmap_v, const PrefillParams p) {
   using Cfg = AttnCfg<D>;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  extern __shared__ __align__(1024) uint8_t smem[];       // the tiles need 1024-byte alignment (128-byte swizzle atoms)
   uint8_t* sQ = smem;
-  uint8_t* sK = sQ + Cfg::kTileBytes;                     // two stages
-  uint8_t* sV = sK + 2 * Cfg::kTileBytes;                 // two stages
-  uint8_t* sP = sV + 2 * Cfg::kTileBytes;
-  AttnBarriers* bars = reinterpret_cast<AttnBarriers*>(sP + 2 * Cfg::kPBytes);   // P is double-buffered
+  constexpr int NS = Cfg::kKvStages;
+  uint8_t* sK = sQ + Cfg::kTileBytes;                     // NS stages
+  uint8_t* sV = sK + NS * Cfg::kTileBytes;                // NS stages
+  AttnBarriers* bars = reinterpret_cast<AttnBarriers*>(sV + NS * Cfg::kTileBytes);
+  float* xch = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 256);   // [2][2][128]: what the two halves of a row exchange
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.z, h = blockIdx.y, g = h / p.group;
@@ -94,18 +112,22 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   const int n_qtiles = (L + kBM - 1) / kBM;
   const int qi = n_qtiles - 1 - static_cast<int>(blockIdx.x);      // the longest rows first
   if (qi < 0) return;                                              // (uniform per CTA, before any barrier)
+  if (smem_u32(smem) & 1023u) {                                    // never seen; would garble every tile
+    if (threadIdx.x == 0) raise_status(p.hdr, FASTKV_ERR_UNSUPPORTED, SITE_ATTN_Q);
+    return;
+  }
   const int q0 = qi * kBM;
   const int n_tiles = qi + 1;                                      // key tiles 0 .. qi (causal)
   const long long limit = p.wait_limit;
 
   if (threadIdx.x == 0) {
     mbar_init(&bars->q_full, 1);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < NS; ++i) {
       mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], 1);
       mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], 1);
-      mbar_init(&bars->s_full[i], 1); mbar_init(&bars->s_free[i], 4);
     }
-    for (int i = 0; i < 2; ++i) { mbar_init(&bars->p_full[i], 4); mbar_init(&bars->p_free[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&bars->s_full[i], 1); mbar_init(&bars->s_free[i], kSoftmaxWarps); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&bars->p_full[i], kSoftmaxWarps); mbar_init(&bars->p_free[i], 1); }
     mbar_init(&bars->o_done, 1);
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -136,15 +158,16 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       bool ok = true;
       int issued = 0;
       for (int j = 0; j < n_tiles && ok; ++j) {
-        const int s = j & 1;
-        ok = mbar_wait_bounded(&bars->k_empty[s], ((j >> 1) & 1) ^ 1, abort_flag, p.hdr, SITE_ATTN_RING, limit);
+        const int s = j % NS;
+        const uint32_t par = (j / NS) & 1;
+        ok = mbar_wait_bounded(&bars->k_empty[s], par ^ 1, abort_flag, p.hdr, SITE_ATTN_RING, limit);
         if (!ok) break;
         mbar_arrive_expect_tx(&bars->k_full[s], Cfg::kTileBytes);
         for (int c = 0; c < Cfg::KH; ++c)
           tma_load_3d(sK + s * Cfg::kTileBytes + c * kChunkBytes, &tmap_k, &bars->k_full[s], c * 64, g, row0 + j * kBN, pol_kv);
-        ok = mbar_wait_bounded(&bars->v_empty[s], ((j >> 1) & 1) ^ 1, abort_flag, p.hdr, SITE_ATTN_RING, limit);
+        ok = mbar_wait_bounded(&bars->v_empty[s], par ^ 1, abort_flag, p.hdr, SITE_ATTN_RING, limit);
         if (!ok) {                                          // K of this tile is in flight, V is not
-          mbar_wait_drain(&bars->k_full[s], (j >> 1) & 1, p.hdr, SITE_ATTN_DRAIN, limit);
+          mbar_wait_drain(&bars->k_full[s], par, p.hdr, SITE_ATTN_DRAIN, limit);
           break;
         }
         mbar_arrive_expect_tx(&bars->v_full[s], Cfg::kTileBytes);
@@ -154,9 +177,9 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       }
       // nothing may still be landing in shared memory when the CTA ends
       mbar_wait_drain(&bars->q_full, 0, p.hdr, SITE_ATTN_DRAIN, limit);
-      for (int j = max(0, issued - 2); j < issued; ++j) {
-        mbar_wait_drain(&bars->k_full[j & 1], (j >> 1) & 1, p.hdr, SITE_ATTN_DRAIN, limit);
-        mbar_wait_drain(&bars->v_full[j & 1], (j >> 1) & 1, p.hdr, SITE_ATTN_DRAIN, limit);
+      for (int j = max(0, issued - NS); j < issued; ++j) {
+        mbar_wait_drain(&bars->k_full[j % NS], (j / NS) & 1, p.hdr, SITE_ATTN_DRAIN, limit);
+        mbar_wait_drain(&bars->v_full[j % NS], (j / NS) & 1, p.hdr, SITE_ATTN_DRAIN, limit);
       }
     }
   } else if (warp == 1) {
@@ -164,40 +187,39 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     if (lane == 0) {
       constexpr uint32_t idesc_s = umma_idesc_bf16_f32(kBM, kBN);
       constexpr uint32_t idesc_o = umma_idesc_bf16_f32(kBM, D) | (1u << 16);      // B (V) is MN-major
-      const uint32_t q_addr = smem_u32(sQ), p_addr = smem_u32(sP);
+      const uint32_t q_addr = smem_u32(sQ);
       bool ok = mbar_wait_bounded(&bars->q_full, 0, abort_flag, p.hdr, SITE_ATTN_Q, limit);
       int committed = 0;
       auto second = [&](int t) {                           // O (+)= P_t V_t
-        const int s = t & 1;
-        ok = mbar_wait_bounded(&bars->v_full[s], (t >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit) &&
-             mbar_wait_bounded(&bars->p_full[s], (t >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_P, limit);
+        const int s = t % NS, pb = t & 1;
+        ok = mbar_wait_bounded(&bars->v_full[s], (t / NS) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit) &&
+             mbar_wait_bounded(&bars->p_full[pb], (t >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_P, limit);
         if (!ok) return;
         tc_fence_after_sync();
         const uint32_t v_addr = smem_u32(sV + s * Cfg::kTileBytes);
 #pragma unroll
-        for (int kk = 0; kk < kBN / 16; ++kk) {
-          const uint64_t adesc = umma_desc_k_sw128(p_addr + s * Cfg::kPBytes + (kk >> 2) * kChunkBytes + (kk & 3) * 32);
+        for (int kk = 0; kk < kBN / 16; ++kk) {            // 16 keys = 8 packed columns of P per step
           const uint64_t bdesc = umma_desc_mn_sw128(v_addr + kk * 2048, kChunkBytes);
-          tc_mma_bf16(tmem_base + 256, adesc, bdesc, idesc_o, (t > 0 || kk > 0) ? 1u : 0u);
+          tc_mma_bf16_ts(tmem_base + 256, tmem_base + 384 + pb * 64 + kk * 8, bdesc, idesc_o, (t > 0 || kk > 0) ? 1u : 0u);
         }
         tc_commit(&bars->v_empty[s]);
-        tc_commit(&bars->p_free[s]);
+        tc_commit(&bars->p_free[pb]);
         ++committed;
       };
       for (int j = 0; j < n_tiles && ok; ++j) {
-        const int s = j & 1;
-        ok = mbar_wait_bounded(&bars->k_full[s], (j >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit) &&
+        const int s = j & 1, ks = j % NS;
+        ok = mbar_wait_bounded(&bars->k_full[ks], (j / NS) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit) &&
              mbar_wait_bounded(&bars->s_free[s], ((j >> 1) & 1) ^ 1, abort_flag, p.hdr, SITE_ATTN_S, limit);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t k_addr = smem_u32(sK + s * Cfg::kTileBytes);
+        const uint32_t k_addr = smem_u32(sK + ks * Cfg::kTileBytes);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint64_t adesc = umma_desc_k_sw128(q_addr + (kk >> 2) * kChunkBytes + (kk & 3) * 32);
           const uint64_t bdesc = umma_desc_k_sw128(k_addr + (kk >> 2) * kChunkBytes + (kk & 3) * 32);
           tc_mma_bf16(tmem_base + s * kBN, adesc, bdesc, idesc_s, kk > 0 ? 1u : 0u);
         }
-        tc_commit(&bars->k_empty[s]);
+        tc_commit(&bars->k_empty[ks]);
         tc_commit(&bars->s_full[s]);
         ++committed;
         if (j >= 1) second(j - 1);
@@ -210,8 +232,9 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       }
     }
   } else {
-    // ---------------- softmax: one query row per thread ----------------
-    const int quarter = warp & 3;
+    // ---------------- softmax: two threads per query row, 64 keys of the tile each ----------------
+    const int gw = warp - 2;
+    const int quarter = warp & 3, half = gw >> 2;         // warps 2..5 and 6..9 cover the four lane quarters once each
     const int r = quarter * 32 + lane;                    // row of the tile = tensor-memory lane
     const int t = q0 + r;                                 // query position in its sequence
     const int t_eff = min(t, L - 1);                      // rows past the end repeat the last row (never stored)
@@ -219,110 +242,121 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     const int jw = t - (L - p.window);                    // window row index, if 0 <= jw < w
     const bool is_window = p.wlog != nullptr && jw >= 0 && t < L;
     float* const wlog_row = is_window ? p.wlog + (static_cast<size_t>(h) * p.window + jw) * p.ld_w + row0 : nullptr;
-    float m_ref = -INFINITY, l = 0.0f;
+    constexpr int HN = kBN / 2;                           // keys per thread and tile
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + (gw & 3)) : "memory"); };
+    float m_ref = -INFINITY, l = 0.0f;                    // the reference is the same in both threads of a row; l is this half's
     bool ok = true;
+    // Both warps of a pair walk every tile and meet at the pair's barrier once per tile whatever happens: a
+    // warp whose wait gave up skips the work of the tile, never the barrier.
     for (int j = 0; j < n_tiles; ++j) {
       const int s = j & 1;
       if (ok) ok = mbar_wait_bounded(&bars->s_full[s], (j >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_SFULL, limit);
       ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after_sync();
-      const int key0 = j * kBN;
-      const bool diagonal = key0 + kBN - 1 > t_eff;       // some keys of the tile are not visible to this row
-      // the whole row of the tile in registers; the S buffer goes back to the issuer at once
-      float v[kBN];
+      const int key0 = j * kBN + half * HN;
+      const bool diagonal = key0 + HN - 1 > t_eff;        // some keys of this half are not visible to this row
+      float v[HN];
+      float half_max = -INFINITY;
+      if (ok) {
+        tc_fence_after_sync();
+        // this half of the row in registers; the S buffer goes back to the issuer at once
 #pragma unroll
-      for (int c = 0; c < kBN / 32; ++c) tmem_ld_32x32(lane_addr + s * kBN + c * 32, *reinterpret_cast<float (*)[32]>(&v[c * 32]));
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->s_free[s]);
-      if (diagonal) {
+        for (int c = 0; c < HN / 32; ++c)
+          tmem_ld_32x32(lane_addr + s * kBN + half * HN + c * 32, *reinterpret_cast<float (*)[32]>(&v[c * 32]));
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->s_free[s]);
+        if (diagonal) {
 #pragma unroll
-        for (int x = 0; x < kBN; ++x) v[x] = key0 + x <= t_eff ? v[x] : -INFINITY;
+          for (int x = 0; x < HN; ++x) v[x] = key0 + x <= t_eff ? v[x] : -INFINITY;
+        }
+        float mx[4] = {v[0], v[1], v[2], v[3]};
+#pragma unroll
+        for (int x = 4; x < HN; x += 4) {
+          mx[0] = fmaxf(mx[0], v[x]); mx[1] = fmaxf(mx[1], v[x + 1]); mx[2] = fmaxf(mx[2], v[x + 2]); mx[3] = fmaxf(mx[3], v[x + 3]);
+        }
+        half_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
       }
-      float mx[4] = {v[0], v[1], v[2], v[3]};
-#pragma unroll
-      for (int x = 4; x < kBN; x += 4) {
-        mx[0] = fmaxf(mx[0], v[x]); mx[1] = fmaxf(mx[1], v[x + 1]); mx[2] = fmaxf(mx[2], v[x + 2]); mx[3] = fmaxf(mx[3], v[x + 3]);
-      }
-      const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;   // the scale is positive
+      xch[(s * 2 + half) * kBM + r] = half_max;
+      pair_sync();
+      if (!ok) continue;
+      const float tile_max = fmaxf(half_max, xch[(s * 2 + (half ^ 1)) * kBM + r]) * p.scale_log2;   // the scale is positive
       // the reference moves only when the tile's maximum is far above it (or at the first tile)
       const bool move = tile_max > m_ref + kRescaleSlackLog2;
       const float alpha = move ? ex2(m_ref - tile_max) : 1.0f;     // 0 at the first tile
       if (move) { m_ref = tile_max; l *= alpha; }
       if (j >= 1 && __any_sync(0xffffffffu, move)) {
-        // O is rescaled once the second contraction of the tile before has been added to it
-        if (ok) ok = mbar_wait_bounded(&bars->p_free[(j - 1) & 1], ((j - 1) >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_PFREE, limit);
+        // O is rescaled (each half its own columns) once the second contraction of the tile before has been added to it
+        ok = mbar_wait_bounded(&bars->p_free[(j - 1) & 1], ((j - 1) >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_PFREE, limit);
         ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
+        if (!ok) continue;
         tc_fence_after_sync();
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
+        for (int c = 0; c < D / 64; ++c) {
           float o[32];
-          tmem_ld_32x32(lane_addr + 256 + c * 32, o);
+          const uint32_t addr = lane_addr + 256 + half * (D / 2) + c * 32;
+          tmem_ld_32x32(addr, o);
 #pragma unroll
           for (int x = 0; x < 32; ++x) o[x] *= alpha;
-          tmem_st_32x32(lane_addr + 256 + c * 32, o);
+          tmem_st_32x32(addr, o);
         }
         tmem_wait_st();
       }
       if (is_window) {                                     // by-product: this row's logits (log2 units), masked = -inf
         float* const dst = wlog_row + key0;
-        if (key0 + kBN <= L && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+        if (key0 + HN <= L && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
 #pragma unroll
-          for (int x = 0; x < kBN; x += 4)
+          for (int x = 0; x < HN; x += 4)
             *reinterpret_cast<float4*>(dst + x) = make_float4(v[x] * p.scale_log2, v[x + 1] * p.scale_log2,
                                                               v[x + 2] * p.scale_log2, v[x + 3] * p.scale_log2);
         } else {
 #pragma unroll
-          for (int x = 0; x < kBN; ++x)
+          for (int x = 0; x < HN; ++x)
             if (key0 + x < L) dst[x] = v[x] * p.scale_log2;
         }
       }
       // this P buffer was last read by the second contraction of tile j - 2
       if (j >= 2) {
-        if (ok) ok = mbar_wait_bounded(&bars->p_free[s], ((j - 2) >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_PFREE, limit);
+        ok = mbar_wait_bounded(&bars->p_free[s], ((j - 2) >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_PFREE, limit);
         ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
+        if (!ok) continue;
       }
-      // p = exp2(s * scale - ref), the row sum, P in bf16 for the second contraction
+      // p = exp2(s * scale - ref), the row sum, P in bf16 for the second contraction: two keys per 32-bit column
+      // of tensor memory, this half's 64 keys in 32 columns of the tile's P buffer
       const float neg_ref = -m_ref;
       float ls[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-      uint8_t* const pbuf = sP + s * Cfg::kPBytes + r * 128;
+      float packed[HN / 2];
 #pragma unroll
-      for (int u = 0; u < kBN / 8; ++u) {                  // 8 keys = 16 bytes per store
-        float e[8];
-#pragma unroll
-        for (int x = 0; x < 8; ++x) {
-          e[x] = ex2(fmaf(v[u * 8 + x], p.scale_log2, neg_ref));      // exp2(-inf) = 0 for a masked key
-          ls[x & 3] += e[x];
-        }
-        uint4 w4;
-        w4.x = pack_bf16(e[0], e[1]);
-        w4.y = pack_bf16(e[2], e[3]);
-        w4.z = pack_bf16(e[4], e[5]);
-        w4.w = pack_bf16(e[6], e[7]);
-        // 16-byte unit (u & 7) of row r sits at unit ((u & 7) ^ (r & 7)) of the row's 128 bytes in its 64-key chunk
-        *reinterpret_cast<uint4*>(pbuf + (u >> 3) * kChunkBytes + (((u & 7) ^ (r & 7)) << 4)) = w4;
+      for (int x = 0; x < HN; x += 2) {
+        const float e0 = ex2(fmaf(v[x], p.scale_log2, neg_ref));      // exp2(-inf) = 0 for a masked key
+        const float e1 = ex2(fmaf(v[x + 1], p.scale_log2, neg_ref));
+        ls[x & 2] += e0;
+        ls[(x & 2) + 1] += e1;
+        packed[x / 2] = __uint_as_float(pack_bf16(e0, e1));
       }
       l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core's proxy
+      tmem_st_32x32(lane_addr + 384 + s * 64 + half * (HN / 2), packed);
+      tmem_wait_st();
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->p_full[s]);
     }
-    // the finished row: O / l -> bf16
+    // the finished row: the halves' sums meet, O / l -> bf16, each half its own columns
+    const int xb = n_tiles & 1;                           // the exchange buffer the last tile did not use
+    xch[(xb * 2 + half) * kBM + r] = l;
+    pair_sync();
+    l += xch[(xb * 2 + (half ^ 1)) * kBM + r];
     if (ok) ok = mbar_wait_bounded(&bars->o_done, 0, abort_flag, p.hdr, SITE_ATTN_ODONE, limit);
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       tc_fence_after_sync();
       const float inv_l = 1.0f / l;
       uint8_t* const orow = reinterpret_cast<uint8_t*>(p.out) +
-                            (static_cast<size_t>(row0 + t) * p.out_stride_tok + static_cast<size_t>(h) * p.out_stride_head) * 2;
+                            (static_cast<size_t>(row0 + t) * p.out_stride_tok + static_cast<size_t>(h) * p.out_stride_head) * 2 +
+                            half * D;                      // D / 2 elements of 2 bytes
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
+      for (int c = 0; c < D / 64; ++c) {
         float o[32];
-        tmem_ld_32x32(lane_addr + 256 + c * 32, o);
+        tmem_ld_32x32(lane_addr + 256 + half * (D / 2) + c * 32, o);
         if (t < L) {
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
@@ -335,7 +369,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           }
         }
       }
-      if (is_window) p.wstat[(static_cast<size_t>(b) * p.n_q_heads + h) * p.window + jw] = make_float2(m_ref, l);
+      if (is_window && half == 0) p.wstat[(static_cast<size_t>(b) * p.n_q_heads + h) * p.window + jw] = make_float2(m_ref, l);
     }
   }
 
