@@ -196,12 +196,13 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
              mbar_wait_bounded(&bars->p_full[pb], (t >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_P, limit);
         if (!ok) return;
         tc_fence_after_sync();
-        const uint32_t v_addr = smem_u32(sV + s * Cfg::kTileBytes);
+        // one descriptor per tile; a step further along K only moves its start-address field (units of 16 bytes)
+        const uint64_t b0 = umma_desc_mn_sw128(smem_u32(sV + s * Cfg::kTileBytes), kChunkBytes);
+        const uint32_t a0 = tmem_base + 384 + pb * 64;
 #pragma unroll
-        for (int kk = 0; kk < kBN / 16; ++kk) {            // 16 keys = 8 packed columns of P per step
-          const uint64_t bdesc = umma_desc_mn_sw128(v_addr + kk * 2048, kChunkBytes);
-          tc_mma_bf16_ts(tmem_base + 256, tmem_base + 384 + pb * 64 + kk * 8, bdesc, idesc_o, (t > 0 || kk > 0) ? 1u : 0u);
-        }
+        for (int kk = 0; kk < kBN / 16; ++kk)              // 16 keys = 8 packed columns of P, 2048 bytes of V per step
+          tc_mma_bf16_ts(tmem_base + 256, a0 + kk * 8, b0 + static_cast<uint64_t>(kk * (2048 >> 4)), idesc_o,
+                         (t > 0 || kk > 0) ? 1u : 0u);
         tc_commit(&bars->v_empty[s]);
         tc_commit(&bars->p_free[pb]);
         ++committed;
@@ -212,12 +213,11 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
              mbar_wait_bounded(&bars->s_free[s], ((j >> 1) & 1) ^ 1, abort_flag, p.hdr, SITE_ATTN_S, limit);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t k_addr = smem_u32(sK + ks * Cfg::kTileBytes);
+        const uint64_t a0 = umma_desc_k_sw128(q_addr), b0 = umma_desc_k_sw128(smem_u32(sK + ks * Cfg::kTileBytes));
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint64_t adesc = umma_desc_k_sw128(q_addr + (kk >> 2) * kChunkBytes + (kk & 3) * 32);
-          const uint64_t bdesc = umma_desc_k_sw128(k_addr + (kk >> 2) * kChunkBytes + (kk & 3) * 32);
-          tc_mma_bf16(tmem_base + s * kBN, adesc, bdesc, idesc_s, kk > 0 ? 1u : 0u);
+        for (int kk = 0; kk < D / 16; ++kk) {              // 64-element chunk kk / 4, 32 bytes per step inside it
+          const uint64_t step = static_cast<uint64_t>(((kk >> 2) * kChunkBytes + (kk & 3) * 32) >> 4);
+          tc_mma_bf16(tmem_base + s * kBN, a0 + step, b0 + step, idesc_s, kk > 0 ? 1u : 0u);
         }
         tc_commit(&bars->k_empty[ks]);
         tc_commit(&bars->s_full[s]);
