@@ -87,6 +87,7 @@ struct Layout {
   int f_rows;                 // un-pooled rows written by pass 2 (KV heads or query heads)
   size_t f_off_counters, f_off_partial, f_off_a, f_zero_bytes, f_bytes;
   int path;                   // the ScorePath fastkv_score takes for this shape; -1: the forced path cannot run it
+  bool partition;             // a batch the parked kernel can score with its sequences side by side
   size_t bytes;               // workspace that path needs
 };
 
@@ -96,6 +97,13 @@ constexpr int kFusedMaxCtas = 148;      // SMs of a B200: one persistent CTA eac
 int parked_tiles_per_cta(int max_len, int ctas) {
   const int ntiles = (max_len + 127) / 128;
   return (ntiles + ctas - 1) / ctas;
+}
+
+// A batch can be scored with its sequences side by side (the parked kernel's partition mode: rounds of
+// sequences that together fit the grid at one ring of tiles per CTA) whenever its longest sequence alone fits.
+// Worth it when the batch has at least about six tiles per CTA and head.
+bool partition_ok(const fastkv_shape& s, int ctas, int slots) {
+  return s.batch >= 2 && s.batch <= 64 && parked_tiles_per_cta(s.max_len, ctas) <= slots;
 }
 
 Layout make_layout(const fastkv_shape& s) {
@@ -143,11 +151,19 @@ Layout make_layout(const fastkv_shape& s) {
   // two-pipeline kernel that reads K a second time from L2 is used; the buffered two-kernel path serves the
   // remaining shapes.
   const int per = parked_tiles_per_cta(s.max_len, kFusedMaxCtas), slots = parked_slots(l.npad);
+  // batches: sequences side by side, in as few rounds as fit the ring (the ring then holds one phase, not two, but
+  // every CTA streams all the time, there are rounds x n_kv_heads phases instead of batch x n_kv_heads, and a
+  // statistics exchange involves the CTAs of one sequence only)
+  const long long batch_per = (static_cast<long long>(s.total_len) / 128 + kFusedMaxCtas - 1) / kFusedMaxCtas;
+  l.partition = partition_ok(s, kFusedMaxCtas, slots);
   switch (g_debug.score_path) {
     case PATH_BUFFERED: l.path = PATH_BUFFERED; break;
     case PATH_REREAD: l.path = l.fused_shape_ok ? PATH_REREAD : PATH_BUFFERED; break;
-    case PATH_PARKED: l.path = !l.fused_shape_ok ? PATH_BUFFERED : (per <= slots ? PATH_PARKED : -1); break;
-    default: l.path = !l.fused_shape_ok ? PATH_BUFFERED : (per >= 6 && 2 * per <= slots ? PATH_PARKED : PATH_REREAD); break;
+    case PATH_PARKED: l.path = !l.fused_shape_ok ? PATH_BUFFERED : (l.partition || per <= slots ? PATH_PARKED : -1); break;
+    default:
+      l.path = !l.fused_shape_ok ? PATH_BUFFERED
+               : (l.partition && batch_per >= 6) || (s.batch == 1 && per >= 6 && 2 * per <= slots) ? PATH_PARKED : PATH_REREAD;
+      break;
   }
   l.bytes = l.path == PATH_BUFFERED ? l.b_bytes : l.f_bytes;
   return l;
@@ -387,7 +403,8 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
     const int ctas = fused_grid();
     if (ctas <= 0) return fail(FASTKV_ERR_UNSUPPORTED, "the device offers no cooperative launch");
     const bool parked = lay.path == PATH_PARKED;
-    if (parked && parked_tiles_per_cta(s.max_len, ctas) > parked_slots(lay.npad))
+    const bool partition = parked && partition_ok(s, ctas, parked_slots(lay.npad));
+    if (parked && !partition && parked_tiles_per_cta(s.max_len, ctas) > parked_slots(lay.npad))
       return fail(FASTKV_ERR_UNSUPPORTED, "this device has too few SMs to park a phase of this length");
     e = parked ? launch_clear_words(ws, lay.f_zero_bytes, stream) : cudaMemsetAsync(ws, 0, lay.f_zero_bytes, stream);
     if (e != cudaSuccess) return cuda_fail(e, "clearing the workspace header");
@@ -415,6 +432,7 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
     fp.max_len = s.max_len;
     fp.wait_limit = g_debug.wait_limit_cycles > 0 ? g_debug.wait_limit_cycles : kWaitLimitCycles;
     fp.extra_publications = g_debug.extra_publications;
+    fp.partition = partition ? 1 : 0;
     {
       TimedLaunch timed(KID_SCORE, stream);
       e = parked ? launch_score_parked(s.head_dim, lay.npad, tmap_k, tmap_q, fp, ctas, stream)

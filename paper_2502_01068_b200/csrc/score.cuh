@@ -57,6 +57,7 @@ struct FusedParams {
   int max_len;                // longest sequence of the batch (host knowledge)
   long long wait_limit;       // cycles a device-side wait may poll before it gives up
   int extra_publications;     // test hook: pass 2 waits for this many publications that never come
+  int partition;              // parked kernel, batch > 1: deal the CTAs out to the sequences (see score_parked.cu)
 };
 
 struct PoolRowsParams {

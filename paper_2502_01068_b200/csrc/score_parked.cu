@@ -4,7 +4,9 @@
 //
 // One persistent CTA per SM (cooperative launch: every CTA is resident).  The work is cut into
 // phases, one per (sequence, KV head); in every phase CTA c owns the same run of consecutive
-// 128-key tiles of the sequence.  Per CTA:
+// 128-key tiles of the sequence.  A batch of several sequences is either walked sequence by sequence
+// by the whole grid, or (partition mode) its sequences are scored side by side, each by its own share
+// of the CTAs.  Per CTA:
 //
 //   producer   one thread streams the K tiles (and the G*w window-query rows of the phase) into a
 //              ring of shared-memory stages with TMA;
@@ -56,6 +58,7 @@ constexpr int kParkedThreads = 32 * (kCtrlWarps + kPass1Warps + kPass2Warps);   
 constexpr int kMaxStages = 8;
 constexpr int kMaxSlots = 16;
 constexpr int kRefBufs = 4;                    // phases whose references may be waiting for pass 2
+constexpr int kMaxBatchPart = 64;              // sequences a partitioned batch may have (rounds <= sequences)
 // Pass 1 keeps e = exp2(s - ref) with the row's first logit as the reference; the reference only moves
 // when a logit exceeds it by more than this many binary orders of magnitude (e and its row sums stay far
 // inside the fp32 range: e <= 2^64, at most 2^20-odd terms per sum).
@@ -72,7 +75,7 @@ struct ParkedCfg {
   static constexpr int kRefBytes = kRefBufs * 4 * NPAD * 4; // one reference per (phase in flight, lane quarter, query row)
   static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 2 * kQBytes + kRefBytes + kBarBytes +
                                     2 * 4 * NPAD * 8 /*warp_stats*/ + NPAD * 8 /*norm*/ +
-                                    2 * kPass2Threads * 8 /*merge_buf*/ + NPAD * 4 /*row_j*/;
+                                    2 * kPass2Threads * 8 /*merge_buf*/ + NPAD * 4 /*row_j*/ + (kMaxBatchPart + 1) * 16 /*part_tab*/;
 };
 
 struct ParkedBarriers {
@@ -141,24 +144,94 @@ __device__ __forceinline__ void add_heads(const float (&pr)[32], float (&a_h)[8]
 // What one CTA does in one phase (one KV head of one sequence).
 struct PhaseWork {
   int b, g, row0, L, t0, n, nact, stat;
+  int slot;        // this CTA's number among the CTAs that share the phase: where its statistics go
 };
 
 struct PhaseIter {
   int b, g;
 };
 
+// Partition mode (a batch whose sequences are scored side by side).  The sequences are taken in rounds of
+// consecutive sequences; within a round the CTAs of the grid are dealt out to the round's sequences in
+// proportion to their length: this CTA is number `cta` of the `ncta` that share sequence b and sees no other
+// sequence of the round.  Every CTA then has tiles in every phase, and a statistics exchange involves only
+// the CTAs of one sequence.  One entry per round, worked out once per CTA and kept in shared memory.
+struct PartEntry {
+  int b;           // the CTA's sequence in this round; kPartIdle: none; kPartEnd: past the last round
+  int cta, ncta;   // its number among the CTAs of that sequence, and how many they are
+  int per;         // tiles per CTA and phase the deal came out at (at most the ring)
+};
+constexpr int kPartIdle = -2, kPartEnd = -3;
+
+__device__ __forceinline__ int seq_tiles(const FusedParams& p, int b) {
+  const int L = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
+  return L < p.window ? 0 : (L + kTileKeys - 1) / kTileKeys;       // a sequence shorter than the window has no scores
+}
+
+// The same arithmetic in every CTA.  Rounds are filled greedily: a sequence joins the round while the round's
+// sequences still fit the grid at `ring` tiles per CTA (one sequence always does: the host checked the
+// longest); inside a round the smallest number of tiles per CTA that fits is used.  Run by one thread.
+__device__ void fill_part_table(const FusedParams& p, int cta, int ncta, int ring, PartEntry* tab) {
+  int b0 = 0, r = 0;
+  while (b0 < p.batch) {
+    int b1 = b0, need = 0, total = 0;
+    while (b1 < p.batch) {
+      const int t = seq_tiles(p, b1), n = (t + ring - 1) / ring;
+      if (b1 > b0 && need + n > ncta) break;
+      need += n;
+      total += t;
+      ++b1;
+    }
+    int per = max(1, (total + ncta - 1) / ncta);
+    while (true) {
+      int n = 0;
+      for (int b = b0; b < b1; ++b) n += (seq_tiles(p, b) + per - 1) / per;
+      if (n <= ncta) break;
+      ++per;
+    }
+    PartEntry e = {kPartIdle, 0, 0, per};                             // a CTA left over in this round
+    int first = 0;
+    for (int b = b0; b < b1; ++b) {
+      const int n = (seq_tiles(p, b) + per - 1) / per;
+      if (cta >= first && cta < first + n) e = {b, cta - first, n, per};
+      first += n;
+    }
+    tab[r++] = e;
+    b0 = b1;
+  }
+  tab[r] = {kPartEnd, 0, 0, 0};
+}
+
 // Every role of every CTA walks the same list of phases with the same arithmetic.
-__device__ __forceinline__ bool next_phase(const FusedParams& p, PhaseIter& it, int cta, int ncta, PhaseWork& w) {
-  if (it.b >= p.batch) return false;
-  w.b = it.b;
-  w.g = it.g;
-  if (++it.g >= p.n_kv_heads) { it.g = 0; ++it.b; }
+template <bool PART>
+__device__ __forceinline__ bool next_phase(const FusedParams& p, PhaseIter& it, int cta, int ncta, const PartEntry* tab,
+                                           PhaseWork& w) {
+  int per_fixed = 0;
+  if (PART) {                                              // the heads of this CTA's sequence, round by round
+    PartEntry e = tab[it.b];                               // (it.b counts rounds here)
+    while (e.b != kPartEnd && (e.b == kPartIdle || it.g >= p.n_kv_heads)) {
+      e = tab[++it.b];
+      it.g = 0;
+    }
+    if (e.b == kPartEnd) return false;
+    w.b = e.b;
+    w.g = it.g++;
+    cta = e.cta;
+    ncta = e.ncta;
+    per_fixed = e.per;
+  } else {
+    if (it.b >= p.batch) return false;
+    w.b = it.b;
+    w.g = it.g;
+    if (++it.g >= p.n_kv_heads) { it.g = 0; ++it.b; }
+  }
+  if (PART) w.slot = cta;
   w.row0 = p.cu_seqlens ? p.cu_seqlens[w.b] : 0;
   w.L = p.cu_seqlens ? p.cu_seqlens[w.b + 1] - w.row0 : p.total_len;
   w.stat = w.b * p.n_kv_heads + w.g;
   if (w.L < p.window) { w.t0 = 0; w.n = 0; w.nact = 0; return true; }
   const int ntiles = (w.L + kTileKeys - 1) / kTileKeys;
-  const int per = (ntiles + ncta - 1) / ncta;
+  const int per = per_fixed > 0 ? per_fixed : (ntiles + ncta - 1) / ncta;
   w.nact = (ntiles + per - 1) / per;
   w.t0 = cta * per;
   w.n = max(0, min(per, ntiles - w.t0));
@@ -171,7 +244,7 @@ static_assert(ParkedCfg<128, 32>::kSmemBytes <= 232448 && ParkedCfg<128, 64>::kS
               ParkedCfg<64, 32>::kSmemBytes <= 232448 && ParkedCfg<64, 64>::kSmemBytes <= 232448,
               "dynamic shared memory per CTA");
 
-template <int D, int NPAD>
+template <int D, int NPAD, bool PART>
 __global__ void __launch_bounds__(kParkedThreads, 1)
 score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_q,
                     const FusedParams p) {
@@ -188,12 +261,18 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
   float2* norm = warp_stats + 2 * 4 * NPAD;                           // [NPAD] (-row max, 1 / row sum)
   float2* merge_buf = norm + NPAD;                                    // [256] partial merges
   int* row_j = reinterpret_cast<int*>(merge_buf + 2 * kPass2Threads); // [NPAD] window row j = n / G of query row n
+  PartEntry* part_tab = reinterpret_cast<PartEntry*>(row_j + NPAD);   // [rounds + 1], partition mode only
   constexpr int CPW = NPAD / 2;                                       // accumulator columns per pass-1 warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, ncta = gridDim.x;
   const long long limit = p.wait_limit;
 
+  if (PART && cta == 0 && threadIdx.x == 0) {
+    // a sequence shorter than the observation window has no defined scores (and no CTA): say so once
+    for (int b = 0; b < p.batch; ++b)
+      if (p.cu_seqlens[b + 1] - p.cu_seqlens[b] < p.window) raise_status(p.hdr, FASTKV_ERR_INVALID_ARG, SITE_SCORE_SHORT_SEQUENCE);
+  }
   // A phase that does not fit in the slot ring could never complete: refuse before any barrier exists.
   if ((((p.max_len + kTileKeys - 1) / kTileKeys) + ncta - 1) / ncta > kSlots) {
     if (cta == 0 && threadIdx.x == 0) raise_status(p.hdr, FASTKV_ERR_UNSUPPORTED, SITE_PARKED_RING);
@@ -214,6 +293,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
       mbar_init(&bars->stats_free[i], 1);
     }
     bars->abort_flag = 0;
+    if (PART) fill_part_table(p, cta, ncta, kSlots, part_tab);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     tma_prefetch_desc(&tmap_k);
@@ -244,7 +324,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
       bool ok = true;
       PhaseIter pit = {0, 0};
       PhaseWork w;
-      while (ok && next_phase(p, pit, cta, ncta, w)) {
+      while (ok && next_phase<PART>(p, pit, cta, ncta, part_tab, w)) {
         if (w.n == 0) continue;
         const int h = u & 1;
         if (u >= 2) ok = mbar_wait_bounded(&bars->q_empty[h], ((u >> 1) - 1) & 1, abort_flag, p.hdr, SITE_FUSED_Q_EMPTY, limit);
@@ -285,7 +365,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
       bool ok = true;
       PhaseIter pit = {0, 0};
       PhaseWork w;
-      while (ok && next_phase(p, pit, cta, ncta, w)) {
+      while (ok && next_phase<PART>(p, pit, cta, ncta, part_tab, w)) {
         if (w.n == 0) continue;
         const int h = u & 1;
         ok = mbar_wait_bounded(&bars->q_full[h], (u >> 1) & 1, abort_flag, p.hdr, SITE_FUSED_Q_FULL, limit);
@@ -322,7 +402,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     bool ok = true;
     PhaseIter pit = {0, 0};
     PhaseWork w;
-    while (next_phase(p, pit, cta, ncta, w)) {
+    while (next_phase<PART>(p, pit, cta, ncta, part_tab, w)) {
       if (w.n == 0) continue;
       const int buf = u & 1;
       if (ok) ok = mbar_wait_bounded(&bars->stats_ready[buf], (u >> 1) & 1, abort_flag, p.hdr, SITE_PARKED_STATS, limit);
@@ -333,7 +413,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         float mm = -INFINITY, ll = 0.0f;
 #pragma unroll
         for (int q = 0; q < 4; ++q) merge_stats(mm, ll, ws[q * NPAD + n].x, ws[q * NPAD + n].y);
-        p.partial[(static_cast<size_t>(w.stat) * ncta + cta) * NPAD + n] = make_float2(mm, ll);
+        p.partial[(static_cast<size_t>(w.stat) * ncta + (PART ? w.slot : cta)) * NPAD + n] = make_float2(mm, ll);
       }
       __syncwarp();
       if (lane == 0) {
@@ -357,7 +437,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     bool ok = true;
     PhaseIter pit = {0, 0};
     PhaseWork w;
-    while (next_phase(p, pit, cta, ncta, w)) {
+    while (next_phase<PART>(p, pit, cta, ncta, part_tab, w)) {
       if (w.n == 0) {
         // a sequence shorter than the observation window has no defined scores: say so once
         if (w.L < p.window && cta == 0 && gw == 0 && lane == 0)
@@ -526,7 +606,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     bool ok = true;
     PhaseIter pit = {0, 0};
     PhaseWork w;
-    while (next_phase(p, pit, cta, ncta, w)) {           // an aborted CTA still walks every phase: see pass2_sync
+    while (next_phase<PART>(p, pit, cta, ncta, part_tab, w)) {           // an aborted CTA still walks every phase: see pass2_sync
       if (w.n == 0) continue;
       const int rbuf = u % kRefBufs;
       {
@@ -674,7 +754,7 @@ cudaError_t launch_clear_words(void* ptr, size_t bytes, cudaStream_t stream) {
   return cudaLaunchKernelEx(&cfg, clear_words_kernel, static_cast<uint32_t*>(ptr), static_cast<int>(bytes / 4));
 }
 
-template <int D, int NPAD>
+template <int D, int NPAD, bool PART>
 static cudaError_t launch_parked_t(const CUtensorMap& tk, const CUtensorMap& tq, const FusedParams& p, int grid,
                                    cudaStream_t stream) {
   using Cfg = ParkedCfg<D, NPAD>;
@@ -683,7 +763,7 @@ static cudaError_t launch_parked_t(const CUtensorMap& tk, const CUtensorMap& tq,
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (!configured.done(dev)) {
-    e = cudaFuncSetAttribute(score_parked_kernel<D, NPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(score_parked_kernel<D, NPAD, PART>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Cfg::kSmemBytes);
     if (e != cudaSuccess) return e;
     configured.set(dev);
@@ -704,22 +784,29 @@ static cudaError_t launch_parked_t(const CUtensorMap& tk, const CUtensorMap& tq,
     fill_pdl_attribute(&attr[1]);
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    e = cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(score_parked_kernel<D, NPAD>), args);
+    e = cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(score_parked_kernel<D, NPAD, PART>), args);
     if (e == cudaSuccess) return e;
     if (e != cudaErrorNotSupported && e != cudaErrorInvalidValue) return e;
     cudaGetLastError();          // the combination is refused: from now on plain cooperative launches
     no_overlap.set(dev);
   }
-  return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(score_parked_kernel<D, NPAD>), dim3(grid),
+  return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(score_parked_kernel<D, NPAD, PART>), dim3(grid),
                                      dim3(kParkedThreads), args, Cfg::kSmemBytes, stream);
 }
 
 cudaError_t launch_score_parked(int head_dim, int npad, const CUtensorMap& tk, const CUtensorMap& tq,
                                 const FusedParams& p, int grid, cudaStream_t stream) {
-  if (head_dim == 128 && npad == 32) return launch_parked_t<128, 32>(tk, tq, p, grid, stream);
-  if (head_dim == 128 && npad == 64) return launch_parked_t<128, 64>(tk, tq, p, grid, stream);
-  if (head_dim == 64 && npad == 32) return launch_parked_t<64, 32>(tk, tq, p, grid, stream);
-  if (head_dim == 64 && npad == 64) return launch_parked_t<64, 64>(tk, tq, p, grid, stream);
+  if (p.partition) {
+    if (head_dim == 128 && npad == 32) return launch_parked_t<128, 32, true>(tk, tq, p, grid, stream);
+    if (head_dim == 128 && npad == 64) return launch_parked_t<128, 64, true>(tk, tq, p, grid, stream);
+    if (head_dim == 64 && npad == 32) return launch_parked_t<64, 32, true>(tk, tq, p, grid, stream);
+    if (head_dim == 64 && npad == 64) return launch_parked_t<64, 64, true>(tk, tq, p, grid, stream);
+    return cudaErrorInvalidValue;
+  }
+  if (head_dim == 128 && npad == 32) return launch_parked_t<128, 32, false>(tk, tq, p, grid, stream);
+  if (head_dim == 128 && npad == 64) return launch_parked_t<128, 64, false>(tk, tq, p, grid, stream);
+  if (head_dim == 64 && npad == 32) return launch_parked_t<64, 32, false>(tk, tq, p, grid, stream);
+  if (head_dim == 64 && npad == 64) return launch_parked_t<64, 64, false>(tk, tq, p, grid, stream);
   return cudaErrorInvalidValue;
 }
 
