@@ -326,6 +326,15 @@ cudaError_t launch_select(const SelectParams& p, int batch, int max_len, cudaStr
   if (max_len <= 2 * 16 * 256) return launch_select_c<2, 256>(p, batch, max_len, stream);
   if (max_len <= 4 * 16 * 256) return launch_select_c<4, 256>(p, batch, max_len, stream);
   if (max_len <= 8 * 16 * 256) return launch_select_c<8, 256>(p, batch, max_len, stream);
+  // Batches: every problem (a score row of a sequence) is a cluster; with many of them, smaller clusters keep the
+  // whole launch in one wave of a 148-SM part (1024-thread CTAs: one per SM) as long as a CTA's share still fits
+  // the register cache (32 candidates per thread): 72 problems x 8 CTAs take four waves, x 2 one.
+  const int problems = (p.set[0].n_rows + p.set[1].n_rows) * batch;
+  int cluster = 8;
+  while (cluster > 1 && problems * cluster > 148 && (max_len + cluster / 2 - 1) / (cluster / 2) <= 32 * 1024) cluster /= 2;
+  if (cluster == 4) return launch_select_c<4, 1024>(p, batch, max_len, stream);
+  if (cluster == 2) return launch_select_c<2, 1024>(p, batch, max_len, stream);
+  if (cluster == 1) return launch_select_c<1, 1024>(p, batch, max_len, stream);
   return launch_select_c<8, 1024>(p, batch, max_len, stream);
 }
 
