@@ -253,6 +253,9 @@ int fastkv_score_static_status(void* stream, int32_t* status, int32_t* site);
  *                         a second time from L2; 3 persistent kernel that parks the logits in
  *                         tensor memory (FASTKV_ERR_UNSUPPORTED from the scoring calls when a
  *                         sequence is too long for it).  fastkv_workspace_bytes follows the choice.
+ *   "score_partition"     path 3: several (sequence, head) phases side by side, each on its share of
+ *                         the CTAs: 0 by shape (batches, and single sequences of middling length);
+ *                         1 never; 2 whenever the shape allows it
  *   "fused_heads"         path 2: KV heads scored side by side in one phase (0: by size)
  *   "fused_lead"          path 2: phases the first read may lead the second (0: by size)
  *   "wait_limit_cycles"   clock cycles a device-side wait of the scoring kernels polls before it

@@ -45,6 +45,7 @@ struct DebugConfig {
   int fused_lead = 0;               // two-pipeline kernel: phases pass 1 may lead pass 2 (0 = by size)
   long long wait_limit_cycles = 0;  // 0 = the default of about a second
   int extra_publications = 0;       // pass 2 waits for publications that never come (timeout test)
+  int score_partition = 0;          // parked kernel's partition mode: 0 = by shape, 1 = never, 2 = whenever it can run
 };
 DebugConfig g_debug;
 
@@ -99,11 +100,11 @@ int parked_tiles_per_cta(int max_len, int ctas) {
   return (ntiles + ctas - 1) / ctas;
 }
 
-// A batch can be scored with its sequences side by side (the parked kernel's partition mode: rounds of
-// sequences that together fit the grid at one ring of tiles per CTA) whenever its longest sequence alone fits.
-// Worth it when the batch has at least about six tiles per CTA and head.
+// The parked kernel's partition mode (several (sequence, head) phases side by side, each on its share of the
+// CTAs, in rounds that fit the grid at one ring of tiles per CTA) can run whenever the longest sequence alone
+// fits the ring and the table of rounds fits its shared memory.
 bool partition_ok(const fastkv_shape& s, int ctas, int slots) {
-  return s.batch >= 2 && s.batch <= 64 && parked_tiles_per_cta(s.max_len, ctas) <= slots;
+  return static_cast<long long>(s.batch) * s.n_kv_heads <= 512 && parked_tiles_per_cta(s.max_len, ctas) <= slots;
 }
 
 Layout make_layout(const fastkv_shape& s) {
@@ -155,14 +156,25 @@ Layout make_layout(const fastkv_shape& s) {
   // every CTA streams all the time, there are rounds x n_kv_heads phases instead of batch x n_kv_heads, and a
   // statistics exchange involves the CTAs of one sequence only)
   const long long batch_per = (static_cast<long long>(s.total_len) / 128 + kFusedMaxCtas - 1) / kFusedMaxCtas;
-  l.partition = partition_ok(s, kFusedMaxCtas, slots);
+  // Partition mode: batches with enough work (sequences x heads exchanges are what it removes: 189 against 266 us
+  // on the ragged config), and single sequences short enough that a grid-wide phase per head leaves CTAs without
+  // tiles, one head per share of the CTAs (kernel alone, re-read / parked / parked with partition: 30.9 / 45.0 /
+  // 27.5 us at 32K, 52.0 / 54.3 / 41.6 at 64K, 83.5 / 61.9 / 59.2 at 96K, 89.9 / 60.8 / 68.3 at 128K; below 24K
+  // the re-read kernel is as fast).
+  const bool partition_wanted = s.batch >= 2 ? batch_per >= 6 : (s.max_len >= 24576 && per <= 6);
+  l.partition = partition_ok(s, kFusedMaxCtas, slots) &&
+                (g_debug.score_partition == 2 || (g_debug.score_partition == 0 && partition_wanted));
   switch (g_debug.score_path) {
     case PATH_BUFFERED: l.path = PATH_BUFFERED; break;
     case PATH_REREAD: l.path = l.fused_shape_ok ? PATH_REREAD : PATH_BUFFERED; break;
-    case PATH_PARKED: l.path = !l.fused_shape_ok ? PATH_BUFFERED : (l.partition || per <= slots ? PATH_PARKED : -1); break;
+    case PATH_PARKED:
+      // forced: batches take the partition mode whenever it can run (the grid-wide walk needs the same ring)
+      if (g_debug.score_partition != 1 && s.batch >= 2 && partition_ok(s, kFusedMaxCtas, slots)) l.partition = true;
+      l.path = !l.fused_shape_ok ? PATH_BUFFERED : (per <= slots ? PATH_PARKED : -1);
+      break;
     default:
       l.path = !l.fused_shape_ok ? PATH_BUFFERED
-               : (l.partition && batch_per >= 6) || (s.batch == 1 && per >= 6 && 2 * per <= slots) ? PATH_PARKED : PATH_REREAD;
+               : l.partition || (s.batch == 1 && per >= 6 && 2 * per <= slots) ? PATH_PARKED : PATH_REREAD;
       break;
   }
   l.bytes = l.path == PATH_BUFFERED ? l.b_bytes : l.f_bytes;
@@ -339,6 +351,9 @@ int fastkv_debug_set(const char* key, int64_t value) {
     g_debug.fused_lead = static_cast<int>(value < 0 ? 0 : value);
   } else if (!std::strcmp(key, "wait_limit_cycles")) {
     g_debug.wait_limit_cycles = value < 0 ? 0 : value;
+  } else if (!std::strcmp(key, "score_partition")) {
+    if (value < 0 || value > 2) return fail(FASTKV_ERR_INVALID_ARG, "debug_set: score_partition is 0..2");
+    g_debug.score_partition = static_cast<int>(value);
   } else if (!std::strcmp(key, "extra_publications")) {
     g_debug.extra_publications = static_cast<int>(value < 0 ? 0 : value);
   } else if (!std::strcmp(key, "time_kernels")) {
@@ -403,7 +418,7 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
     const int ctas = fused_grid();
     if (ctas <= 0) return fail(FASTKV_ERR_UNSUPPORTED, "the device offers no cooperative launch");
     const bool parked = lay.path == PATH_PARKED;
-    const bool partition = parked && partition_ok(s, ctas, parked_slots(lay.npad));
+    const bool partition = parked && lay.partition && partition_ok(s, ctas, parked_slots(lay.npad));
     if (parked && !partition && parked_tiles_per_cta(s.max_len, ctas) > parked_slots(lay.npad))
       return fail(FASTKV_ERR_UNSUPPORTED, "this device has too few SMs to park a phase of this length");
     e = parked ? launch_clear_words(ws, lay.f_zero_bytes, stream) : cudaMemsetAsync(ws, 0, lay.f_zero_bytes, stream);
@@ -432,7 +447,7 @@ int fastkv_score(const fastkv_shape* shape, const void* q, const void* k, float*
     fp.max_len = s.max_len;
     fp.wait_limit = g_debug.wait_limit_cycles > 0 ? g_debug.wait_limit_cycles : kWaitLimitCycles;
     fp.extra_publications = g_debug.extra_publications;
-    fp.partition = partition ? 1 : 0;
+    fp.partition = partition ? (s.batch >= 2 ? 1 : 2) : 0;
     {
       TimedLaunch timed(KID_SCORE, stream);
       e = parked ? launch_score_parked(s.head_dim, lay.npad, tmap_k, tmap_q, fp, ctas, stream)

@@ -57,7 +57,8 @@ struct FusedParams {
   int max_len;                // longest sequence of the batch (host knowledge)
   long long wait_limit;       // cycles a device-side wait may poll before it gives up
   int extra_publications;     // test hook: pass 2 waits for this many publications that never come
-  int partition;              // parked kernel, batch > 1: deal the CTAs out to the sequences (see score_parked.cu)
+  int partition;              // parked kernel: 0 the grid walks the phases together; 1 CTAs dealt out to the sequences
+                              // of a batch; 2 to the (sequence, head) pairs (see score_parked.cu)
 };
 
 struct PoolRowsParams {

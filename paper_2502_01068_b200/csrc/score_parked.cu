@@ -4,8 +4,8 @@
 //
 // One persistent CTA per SM (cooperative launch: every CTA is resident).  The work is cut into
 // phases, one per (sequence, KV head); in every phase CTA c owns the same run of consecutive
-// 128-key tiles of the sequence.  A batch of several sequences is either walked sequence by sequence
-// by the whole grid, or (partition mode) its sequences are scored side by side, each by its own share
+// 128-key tiles of the sequence.  Either the whole grid walks the phases one after the other, or
+// (partition mode: batches, short sequences) several phases run side by side, each on its own share
 // of the CTAs.  Per CTA:
 //
 //   producer   one thread streams the K tiles (and the G*w window-query rows of the phase) into a
@@ -58,7 +58,7 @@ constexpr int kParkedThreads = 32 * (kCtrlWarps + kPass1Warps + kPass2Warps);   
 constexpr int kMaxStages = 8;
 constexpr int kMaxSlots = 16;
 constexpr int kRefBufs = 4;                    // phases whose references may be waiting for pass 2
-constexpr int kMaxBatchPart = 64;              // sequences a partitioned batch may have (rounds <= sequences)
+constexpr int kMaxPartUnits = 512;             // (sequence, KV head) pairs a partitioned launch may have (rounds <= units)
 // Pass 1 keeps e = exp2(s - ref) with the row's first logit as the reference; the reference only moves
 // when a logit exceeds it by more than this many binary orders of magnitude (e and its row sums stay far
 // inside the fp32 range: e <= 2^64, at most 2^20-odd terms per sum).
@@ -75,7 +75,7 @@ struct ParkedCfg {
   static constexpr int kRefBytes = kRefBufs * 4 * NPAD * 4; // one reference per (phase in flight, lane quarter, query row)
   static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 2 * kQBytes + kRefBytes + kBarBytes +
                                     2 * 4 * NPAD * 8 /*warp_stats*/ + NPAD * 8 /*norm*/ +
-                                    2 * kPass2Threads * 8 /*merge_buf*/ + NPAD * 4 /*row_j*/ + (kMaxBatchPart + 1) * 16 /*part_tab*/;
+                                    2 * kPass2Threads * 8 /*merge_buf*/ + NPAD * 4 /*row_j*/ + (kMaxPartUnits + 1) * 20 /*part_tab*/;
 };
 
 struct ParkedBarriers {
@@ -151,55 +151,61 @@ struct PhaseIter {
   int b, g;
 };
 
-// Partition mode (a batch whose sequences are scored side by side).  The sequences are taken in rounds of
-// consecutive sequences; within a round the CTAs of the grid are dealt out to the round's sequences in
-// proportion to their length: this CTA is number `cta` of the `ncta` that share sequence b and sees no other
-// sequence of the round.  Every CTA then has tiles in every phase, and a statistics exchange involves only
-// the CTAs of one sequence.  One entry per round, worked out once per CTA and kept in shared memory.
+// Partition mode.  Units of work -- a whole sequence (all its KV heads, one after the other: p.partition == 1,
+// batches) or one KV head of a sequence (p.partition == 2, a single sequence of middling length) -- are taken
+// in rounds of consecutive units; within a round the CTAs of the grid are dealt out to the round's units in
+// proportion to their length: this CTA is number `cta` of the `ncta` that share the unit and sees no other
+// unit of the round.  The units of a round are scored side by side, every CTA has tiles in every phase, and a
+// statistics exchange involves only the CTAs of one unit.  That is what batches and shorter sequences want (a
+// grid-wide phase per head would cost sequences x heads exchanges, or leave most CTAs without a tile); a
+// single long sequence is better off with the whole grid on one head at a time and two phases in the ring.
+// One entry per round, worked out once per CTA and kept in shared memory.
 struct PartEntry {
-  int b;           // the CTA's sequence in this round; kPartIdle: none; kPartEnd: past the last round
-  int cta, ncta;   // its number among the CTAs of that sequence, and how many they are
-  int per;         // tiles per CTA and phase the deal came out at (at most the ring)
+  int b, g;        // the CTA's unit in this round (g < 0: every head of b in turn); b == kPartIdle: none; kPartEnd: no more rounds
+  int cta, ncta;   // its number among the CTAs of that unit, and how many they are
+  int per;         // tiles per CTA the deal came out at (at most the ring)
 };
 constexpr int kPartIdle = -2, kPartEnd = -3;
 
 __device__ __forceinline__ int seq_tiles(const FusedParams& p, int b) {
-  const int L = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
+  const int row0 = p.cu_seqlens ? p.cu_seqlens[b] : 0;
+  const int L = p.cu_seqlens ? p.cu_seqlens[b + 1] - row0 : p.total_len;
   return L < p.window ? 0 : (L + kTileKeys - 1) / kTileKeys;       // a sequence shorter than the window has no scores
 }
 
-// The same arithmetic in every CTA.  Rounds are filled greedily: a sequence joins the round while the round's
-// sequences still fit the grid at `ring` tiles per CTA (one sequence always does: the host checked the
-// longest); inside a round the smallest number of tiles per CTA that fits is used.  Run by one thread.
+// The same arithmetic in every CTA.  Rounds are filled greedily: a unit joins the round while the round's
+// units still fit the grid at `ring` tiles per CTA (one unit always does: the host checked the longest
+// sequence); inside a round the smallest number of tiles per CTA that fits is used.  Run by one thread.
 __device__ void fill_part_table(const FusedParams& p, int cta, int ncta, int ring, PartEntry* tab) {
-  int b0 = 0, r = 0;
-  while (b0 < p.batch) {
-    int b1 = b0, need = 0, total = 0;
-    while (b1 < p.batch) {
-      const int t = seq_tiles(p, b1), n = (t + ring - 1) / ring;
-      if (b1 > b0 && need + n > ncta) break;
+  const int H = p.partition == 2 ? p.n_kv_heads : 1, units = p.batch * H;
+  int u0 = 0, r = 0;
+  while (u0 < units) {
+    int u1 = u0, need = 0, total = 0;
+    while (u1 < units) {
+      const int t = seq_tiles(p, u1 / H), n = (t + ring - 1) / ring;
+      if (u1 > u0 && need + n > ncta) break;
       need += n;
       total += t;
-      ++b1;
+      ++u1;
     }
     int per = max(1, (total + ncta - 1) / ncta);
     while (true) {
       int n = 0;
-      for (int b = b0; b < b1; ++b) n += (seq_tiles(p, b) + per - 1) / per;
+      for (int u = u0; u < u1; ++u) n += (seq_tiles(p, u / H) + per - 1) / per;
       if (n <= ncta) break;
       ++per;
     }
-    PartEntry e = {kPartIdle, 0, 0, per};                             // a CTA left over in this round
+    PartEntry e = {kPartIdle, 0, 0, 0, per};                          // a CTA left over in this round
     int first = 0;
-    for (int b = b0; b < b1; ++b) {
-      const int n = (seq_tiles(p, b) + per - 1) / per;
-      if (cta >= first && cta < first + n) e = {b, cta - first, n, per};
+    for (int u = u0; u < u1; ++u) {
+      const int n = (seq_tiles(p, u / H) + per - 1) / per;
+      if (cta >= first && cta < first + n) e = {u / H, p.partition == 2 ? u % H : -1, cta - first, n, per};
       first += n;
     }
     tab[r++] = e;
-    b0 = b1;
+    u0 = u1;
   }
-  tab[r] = {kPartEnd, 0, 0, 0};
+  tab[r] = {kPartEnd, 0, 0, 0, 0};
 }
 
 // Every role of every CTA walks the same list of phases with the same arithmetic.
@@ -207,15 +213,16 @@ template <bool PART>
 __device__ __forceinline__ bool next_phase(const FusedParams& p, PhaseIter& it, int cta, int ncta, const PartEntry* tab,
                                            PhaseWork& w) {
   int per_fixed = 0;
-  if (PART) {                                              // the heads of this CTA's sequence, round by round
+  if (PART) {                                              // this CTA's unit of the round: one head, or all heads in turn
     PartEntry e = tab[it.b];                               // (it.b counts rounds here)
-    while (e.b != kPartEnd && (e.b == kPartIdle || it.g >= p.n_kv_heads)) {
+    while (e.b == kPartIdle || (e.b >= 0 && it.g >= (e.g < 0 ? p.n_kv_heads : 1))) {
       e = tab[++it.b];
       it.g = 0;
     }
     if (e.b == kPartEnd) return false;
     w.b = e.b;
-    w.g = it.g++;
+    w.g = e.g < 0 ? it.g : e.g;
+    ++it.g;
     cta = e.cta;
     ncta = e.ncta;
     per_fixed = e.per;
@@ -271,7 +278,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
   if (PART && cta == 0 && threadIdx.x == 0) {
     // a sequence shorter than the observation window has no defined scores (and no CTA): say so once
     for (int b = 0; b < p.batch; ++b)
-      if (p.cu_seqlens[b + 1] - p.cu_seqlens[b] < p.window) raise_status(p.hdr, FASTKV_ERR_INVALID_ARG, SITE_SCORE_SHORT_SEQUENCE);
+      if (seq_tiles(p, b) == 0) raise_status(p.hdr, FASTKV_ERR_INVALID_ARG, SITE_SCORE_SHORT_SEQUENCE);
   }
   // A phase that does not fit in the slot ring could never complete: refuse before any barrier exists.
   if ((((p.max_len + kTileKeys - 1) / kTileKeys) + ncta - 1) / ncta > kSlots) {

@@ -141,6 +141,18 @@ def test_batch_scored_side_by_side_in_several_rounds(debug_hooks):
     check_layer(wl, x, gpu_layer(wl, x), o, what="five sequences, parked kernel")
 
 
+@pytest.mark.parametrize("L", [700, 40000, 100000])
+def test_single_sequence_with_its_heads_side_by_side(debug_hooks, L):
+    """The parked kernel with one KV head per share of the CTAs (what the library picks for 24K .. 113K tokens at
+    the 8B head shape), forced on short, middling and long single sequences; G = 2, four KV heads."""
+    debug_hooks("score_path", 3)
+    debug_hooks("score_partition", 2)
+    wl = small("heads_side_by_side", 604, [L], [2000 if L > 2000 else 300], [4000 if L > 4000 else 200], Hq=8, Hkv=4, d=64, hidden=64)
+    x = W.make_layer(wl)
+    for order in (B.GROUP_THEN_POOL, B.POOL_THEN_GROUP):
+        check_layer(wl, x, gpu_layer(wl, x, agg_order=order), oracle_layer(wl, x, agg_order=order), what="L=%d order %d" % (L, order))
+
+
 @pytest.mark.parametrize("path", [2, 3])
 def test_group_sizes_and_wide_windows_on_the_persistent_kernels(debug_hooks, path):
     debug_hooks("score_path", path)
