@@ -46,6 +46,7 @@ struct DebugConfig {
   long long wait_limit_cycles = 0;  // 0 = the default of about a second
   int extra_publications = 0;       // pass 2 waits for publications that never come (timeout test)
   int score_partition = 0;          // parked kernel's partition mode: 0 = by shape, 1 = never, 2 = whenever it can run
+  int prefill_skip_commit = 0;      // prefill attention: n > 0: key tile n - 1's "P consumed" signal is withheld (timeout test)
 };
 DebugConfig g_debug;
 
@@ -354,6 +355,8 @@ int fastkv_debug_set(const char* key, int64_t value) {
   } else if (!std::strcmp(key, "score_partition")) {
     if (value < 0 || value > 2) return fail(FASTKV_ERR_INVALID_ARG, "debug_set: score_partition is 0..2");
     g_debug.score_partition = static_cast<int>(value);
+  } else if (!std::strcmp(key, "prefill_skip_commit")) {
+    g_debug.prefill_skip_commit = static_cast<int>(value < 0 ? 0 : value);
   } else if (!std::strcmp(key, "extra_publications")) {
     g_debug.extra_publications = static_cast<int>(value < 0 ? 0 : value);
   } else if (!std::strcmp(key, "time_kernels")) {
@@ -760,6 +763,7 @@ int fastkv_prefill_attention(const fastkv_shape* shape, const void* q, const voi
   pp.wstat = reinterpret_cast<float2*>(ws + lay.off_wstat);
   pp.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
   pp.wait_limit = g_debug.wait_limit_cycles > 0 ? g_debug.wait_limit_cycles : kWaitLimitCycles;
+  pp.skip_commit_tile = g_debug.prefill_skip_commit - 1;
   {
     TimedLaunch timed(KID_PREFILL, stream);
     e = launch_prefill_attn(s.head_dim, tmap_q, tmap_k, tmap_v, pp, s.max_len, stream);

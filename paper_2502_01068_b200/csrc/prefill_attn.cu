@@ -204,7 +204,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           tc_mma_bf16_ts(tmem_base + 256, a0 + kk * 8, b0 + static_cast<uint64_t>(kk * (2048 >> 4)), idesc_o,
                          (t > 0 || kk > 0) ? 1u : 0u);
         tc_commit(&bars->v_empty[s]);
-        tc_commit(&bars->p_free[pb]);
+        if (t != p.skip_commit_tile) tc_commit(&bars->p_free[pb]);     // (test hook: a completion that is never signalled)
         ++committed;
       };
       for (int j = 0; j < n_tiles && ok; ++j) {

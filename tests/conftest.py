@@ -30,7 +30,8 @@ def pytest_collection_modifyitems(config, items):
 def debug_hooks():
     """Sets the library's process-wide test hooks for one test and puts the defaults back afterwards."""
     from paper_2502_01068_b200 import binding as B
-    keys = ("score_path", "score_partition", "fused_heads", "fused_lead", "wait_limit_cycles", "extra_publications")
+    keys = ("score_path", "score_partition", "fused_heads", "fused_lead", "wait_limit_cycles", "extra_publications",
+            "prefill_skip_commit")
 
     def set_hook(key, value):
         assert key in keys

@@ -42,3 +42,41 @@ def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_correct(debug_hoo
     o = oracle_layer(wl, x)
     check_layer(wl, x, g, o, what="after the timeout")
     np.testing.assert_allclose(s_kv.cpu().numpy(), o["S_kv"], rtol=2e-3, atol=1e-12)
+
+
+SITE_ATTN_P_CONSUMED_WAIT = 34       # the softmax warps' wait for "P of the tile two before was consumed"
+SITE_ATTN_P_READY_WAIT = 31          # the issuer's wait for the P the stalled softmax warps never hand over
+
+
+def test_prefill_attention_wait_that_runs_out(debug_hooks):
+    """The prefill attention's softmax warps wait (bounded) for the tensor core to have consumed P of the tile two
+    before; the test hook withholds that signal for one key tile.  The wait gives up after about two milliseconds,
+    every role of the CTA runs out of its loops, copies and contractions in flight are waited for, the status word
+    says where -- and the next call on the same workspace is correct."""
+    import oracle
+    wl = W.Workload(name="prefill_timeout", cfg=980, n_q_heads=4, n_kv_heads=2, head_dim=64, hidden_dim=64, window=8,
+                    pool_kernel=7, pool_mode=W.POOL_AVG, seq_lens=[900], k_kv=[8], k_tsp=[8])
+    x = W.make_layer(wl)
+    q_full = W.full_q(wl, x)
+    L = wl.total_len
+    shape = B.make_shape(total_len=L, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim,
+                         window=wl.window, pool_kernel=wl.pool_kernel, q_layout=B.Q_FULL)
+    ws = torch.empty(B.fastkv_prefill_workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+    out = torch.zeros((L, wl.n_q_heads, wl.head_dim), dtype=torch.int16, device="cuda")
+    s_kv = torch.zeros((wl.n_kv_heads, L), dtype=torch.float32, device="cuda")
+    debug_hooks("wait_limit_cycles", 1 << 22)
+    debug_hooks("prefill_skip_commit", 2)                      # key tile 1: query tiles with four or more key tiles stall
+    B.fastkv_prefill_attention(shape, dev(q_full), dev(x.k), dev(x.v), out, s_kv, None, ws)
+    status, site = B.fastkv_device_status(ws)
+    assert status == B.ERR_DEVICE_TIMEOUT
+    assert site in (SITE_ATTN_P_CONSUMED_WAIT, SITE_ATTN_P_READY_WAIT)       # whichever of the two polls longer first
+
+    debug_hooks("wait_limit_cycles", 0)
+    debug_hooks("prefill_skip_commit", 0)
+    B.fastkv_prefill_attention(shape, dev(q_full), dev(x.k), dev(x.v), out, s_kv, None, ws)
+    assert B.fastkv_device_status(ws) == (0, 0)
+    got = W.bf16_bits_to_f32(out.cpu().numpy().view(np.uint16)).astype(np.float64)
+    ref = oracle.prefill_attention(q_full, x.k, x.v)
+    assert np.all(np.abs(got - ref) <= 1e-2 * np.abs(ref) + 1e-2)
+    o = oracle_layer(wl, x, do_compact=False)
+    np.testing.assert_allclose(s_kv.cpu().numpy(), o["S_kv"], rtol=2e-3, atol=1e-12)
