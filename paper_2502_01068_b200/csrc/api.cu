@@ -146,12 +146,13 @@ Layout make_layout(const fastkv_shape& s) {
   l.f_off_a = off;
   off += round_up(sizeof(float) * static_cast<size_t>(l.f_rows) * l.ld_logits, 256);
   l.f_bytes = off;
-  // Which kernel scores this shape.  The parked kernel is the fastest for long sequences, as long as a CTA's
-  // tiles of two phases fit in its tensor-memory ring (measured on a B200 with the Llama-3.1-8B head shape:
-  // 64 us against 89 us at 131072 tokens); it pays a few microseconds per phase, so below about six tiles per
-  // CTA and phase (57 us against 51 us at 65536 tokens, 37 against 18 at 8192), and beyond the ring, the
-  // two-pipeline kernel that reads K a second time from L2 is used; the buffered two-kernel path serves the
-  // remaining shapes.
+  // Which kernel scores this shape (measured on a B200 with the Llama-3.1-8B head shape, kernel alone, re-read /
+  // parked / parked with partition, us: 17.9 / 35.0 / 18.7 at 8K, 30.9 / 45.0 / 27.5 at 32K, 52.0 / 54.3 / 41.6 at
+  // 64K, 83.5 / 61.9 / 59.2 at 96K, 89.9 / 60.8 / 68.3 at 128K, 122.9 / 90.0 / 96.8 at 200K, 180.9 / 131.8 / 137.7 at
+  // 300K).  A single sequence: below 24K tokens the kernel that reads K a second time from L2 (no per-phase
+  // exchange to pay); up to six tiles per CTA and head the parked kernel with its heads side by side; up to the
+  // ring (16 tiles per CTA: 303K tokens) the parked kernel with the whole grid on one head at a time; beyond the
+  // ring the re-read kernel again.  Batches: see below.  The buffered two-kernel path serves the remaining shapes.
   const int per = parked_tiles_per_cta(s.max_len, kFusedMaxCtas), slots = parked_slots(l.npad);
   // batches: sequences side by side, in as few rounds as fit the ring (the ring then holds one phase, not two, but
   // every CTA streams all the time, there are rounds x n_kv_heads phases instead of batch x n_kv_heads, and a
@@ -175,7 +176,7 @@ Layout make_layout(const fastkv_shape& s) {
       break;
     default:
       l.path = !l.fused_shape_ok ? PATH_BUFFERED
-               : l.partition || (s.batch == 1 && per >= 6 && 2 * per <= slots) ? PATH_PARKED : PATH_REREAD;
+               : l.partition || (s.batch == 1 && per >= 7 && per <= slots) ? PATH_PARKED : PATH_REREAD;
       break;
   }
   l.bytes = l.path == PATH_BUFFERED ? l.b_bytes : l.f_bytes;

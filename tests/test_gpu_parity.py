@@ -101,15 +101,16 @@ def test_every_scoring_kernel_matches(debug_hooks, path):
 
 
 def test_sequence_longer_than_half_the_tensor_memory_ring(debug_hooks):
-    """L = 160 000: a CTA would own 9 tiles per phase, more than half of the 16 parked slots, so the
-    library picks the kernel that re-reads K from L2 by itself; the parked kernel, forced, still works
-    (9 <= 16) and gives the same result up to rounding."""
+    """L = 160 000: a CTA owns 9 tiles per phase, more than half of the 16 parked slots, so the statistics of a
+    phase cannot hide behind a whole next phase; the library still picks the parked kernel (it is the faster one up
+    to the ring), and every scoring kernel, forced, gives the same result up to rounding."""
     wl = small("long", 601, [160000], [4000], [8000], Hq=4, Hkv=1, d=64, hidden=64)
     x = W.make_layer(wl)
     o = oracle_layer(wl, x)
     check_layer(wl, x, gpu_layer(wl, x), o, what="160k")
-    debug_hooks("score_path", 3)
-    check_layer(wl, x, gpu_layer(wl, x), o, what="160k parked")
+    for path in (3, 2):
+        debug_hooks("score_path", path)
+        check_layer(wl, x, gpu_layer(wl, x), o, what="160k, path %d" % path)
 
 
 def test_parked_kernel_at_the_edge_of_its_ring(debug_hooks):
