@@ -137,6 +137,7 @@ def make_shape(*, total_len: int, n_q_heads: int, n_kv_heads: int, head_dim: int
     s.window, s.pool_kernel, s.pool_mode, s.agg_order = window, pool_kernel, pool_mode, agg_order
     s.force_window, s.q_layout, s.softmax_scale = int(force_window), q_layout, softmax_scale
     s.cu_seqlens = _p(cu_seqlens)
+    s._keep_alive = cu_seqlens          # the struct only holds the address: the tensor must outlive it
     s.q_stride_head = head_dim if q_stride_head is None else q_stride_head
     s.q_stride_tok = n_q_heads * head_dim if q_stride_tok is None else q_stride_tok
     s.k_stride_head = head_dim if k_stride_head is None else k_stride_head
@@ -151,6 +152,7 @@ def make_budget(k: int = 0, *, batch: int = 1, cu_k=None, total: Optional[int] =
     b = Budget()
     b.k = k
     b.cu_k = _p(cu_k)
+    b._keep_alive = cu_k                # the struct only holds the address: the tensor must outlive it
     b.total = (k * batch) if total is None else total
     return b
 
