@@ -276,6 +276,134 @@ def oracle_baseline(name: str, wl: W.Workload, x: W.LayerInputs, budget_s: float
     return out
 
 
+LAYER_SEQUENCES = {
+    # config 3: layers 0..14 on the full prompt (KV selection only), Token-Selective Propagation at layer 15,
+    # layers 16..31 on the propagated tokens with the KV budget of the original prompt
+    "llama8b_32k_sweep": lambda: [("layers 0-14 (L = 32768, KV only)", 15, W.llama8b_32k_sweep(), False, None),
+                                  ("layer 15 (L = 32768, TSP)", 1, W.llama8b_32k_sweep(), True, None),
+                                  ("layers 16-31 (L = 6553, KV only)", 16, W.llama8b_32k_sweep(), False, 6553)],
+    # config 4: the layer after the TSP layer runs on the 26214 propagated tokens and keeps 13107 of them
+    "llama8b_128k_post_tsp_layer": lambda: [("post-TSP layer (L = 26214, KV only)", 1, W.llama8b_128k(), False, 26214)],
+}
+
+
+def run_layer_sequence(args) -> None:
+    """A sequence of layers of different kinds (the 32-layer sweep of config 3, the post-TSP layer of config 4):
+    every kind is timed by itself like the default workload's step -- CUDA events on the launching stream,
+    the L2 overwritten before every step because these inputs fit in it, the L2-warm figure beside it,
+    per-kernel times from the library's hook -- and `ms_per_step` is the sum over the sequence."""
+    import dataclasses
+    import torch
+    from paper_2502_01068_b200 import binding as B
+    torch.cuda.set_device(0)
+    stream = torch.cuda.current_stream()
+    warmup, steps = max(3, args.warmup), max(1, min(args.steps, 50))
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    tdev = lambda a: torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).cuda()
+    peaks = measured_peaks()
+    sampler = ClockSampler(0)
+    sampler.start()
+    n0 = B.fastkv_kernel_launches()
+    kinds, total_ms, total_warm, total_tokens, total_bytes = [], 0.0, 0.0, 0, 0
+    kernel_tot = {}
+    for label, count, wl, with_tsp, length in LAYER_SEQUENCES[args.workload]():
+        if length is not None:
+            wl = dataclasses.replace(wl, seq_lens=[length])
+        if not with_tsp:
+            wl = dataclasses.replace(wl, k_tsp=None)
+        wl = dataclasses.replace(wl, k_kv=[min(wl.k_kv[0], wl.seq_lens[0])])
+        x = W.make_layer(wl, with_hidden=with_tsp)
+        L = wl.total_len
+        shape = B.make_shape(total_len=L, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim,
+                             hidden_dim=wl.hidden_dim, window=wl.window, pool_kernel=wl.pool_kernel, pool_mode=wl.pool_mode)
+        q, k, v = tdev(x.q_win), tdev(x.k), tdev(x.v)
+        b_kv = B.make_budget(int(wl.k_kv[0]))
+        ws = torch.empty(B.fastkv_workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+        s_kv = torch.empty((wl.n_kv_heads, L), dtype=torch.float32, device="cuda")
+        idx_kv = torch.empty((wl.n_kv_heads, b_kv.total), dtype=torch.int32, device="cuda")
+        k_out = torch.empty((wl.n_kv_heads, b_kv.total, wl.head_dim), dtype=torch.int16, device="cuda")
+        v_out = torch.empty_like(k_out)
+        if with_tsp:
+            hid, pos = tdev(x.hidden), tdev(x.pos)
+            b_tsp = B.make_budget(int(wl.k_tsp[0]))
+            s_tsp = torch.empty((L,), dtype=torch.float32, device="cuda")
+            idx_tsp = torch.empty((b_tsp.total,), dtype=torch.int32, device="cuda")
+            hid_out = torch.empty((b_tsp.total, wl.hidden_dim), dtype=torch.int16, device="cuda")
+            pos_out = torch.empty((b_tsp.total,), dtype=torch.int32, device="cuda")
+
+            def step():
+                B.fastkv_score(shape, q, k, s_kv, s_tsp, ws, stream)
+                B.fastkv_select(shape, s_kv, b_kv, idx_kv, s_tsp, b_tsp, idx_tsp, ws, stream)
+                B.fastkv_compact(shape, idx_kv, b_kv, idx_tsp, b_tsp, k, v, hid, pos, k_out, v_out, hid_out, pos_out, ws, stream)
+        else:
+            def step():
+                B.fastkv_score(shape, q, k, s_kv, None, ws, stream)
+                B.fastkv_select_kv(shape, s_kv, b_kv, idx_kv, ws, stream)
+                B.fastkv_compact(shape, idx_kv, b_kv, None, None, k, v, None, None, k_out, v_out, None, None, ws, stream)
+
+        for _ in range(warmup):
+            step()
+        torch.cuda.synchronize()
+        status, site = B.fastkv_device_status(ws)
+        if status != 0:
+            raise SystemExit("device status %d at site %d (%s)" % (status, site, label))
+
+        def timed(with_flush: bool) -> float:
+            ts = []
+            for _ in range(steps):
+                if with_flush:
+                    flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                step()
+                e1.record(stream)
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            return statistics.median(ts)
+
+        ms, ms_warm = timed(True), timed(False)
+        B.fastkv_debug_set("time_kernels", 1)
+        for _ in range(steps):
+            flush.zero_()
+            step()
+        torch.cuda.synchronize()
+        B.fastkv_debug_set("time_kernels", 0)
+        kernel_ms = {}
+        for kid, kname in KERNELS.items():
+            _name, kms, cnt = B.fastkv_debug_kernel_time(kid)
+            if cnt:
+                kernel_ms[kname] = kms / cnt
+                kernel_tot[kname] = kernel_tot.get(kname, 0.0) + count * kms / cnt
+        ab = algorithmic_bytes(wl)
+        kinds.append({"layers": label, "count": count, "tokens": L, "k_kv": int(wl.k_kv[0]),
+                      "k_tsp": int(wl.k_tsp[0]) if with_tsp else None, "ms": ms, "ms_l2_warm": ms_warm,
+                      "kernels_ms": kernel_ms, "bytes_rw": ab["step_rw"],
+                      "frac_of_measured": ab["step_rw"] / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]})
+        total_ms += count * ms
+        total_warm += count * ms_warm
+        total_tokens += count * L
+        total_bytes += count * ab["step_rw"]
+    launches = B.fastkv_kernel_launches() - n0
+    clocks = sampler.stop()
+    dominant = max(kernel_tot, key=kernel_tot.get)
+    gbs = total_bytes / (total_ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": total_tokens / (total_ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
+        "warmup": warmup, "ms_per_step": total_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "step": "every layer of the sequence once (sum of count x median time of its kind)",
+                   "n_q_heads": 32, "n_kv_heads": 8, "head_dim": 128, "hidden_dim": 4096, "window": 8, "pool_kernel": 7,
+                   "l2": "L2 overwritten (256 MB write) before every step, not timed: these inputs fit in L2"},
+        "clocks": clocks, "gpu_launches": int(launches), "e2e": None,
+        "roofline": {"bound": "hbm", "kernel": KERNEL_SYMBOLS[dominant], "achieved": gbs, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                     "algorithmic_bytes": total_bytes, "traffic": None,
+                     "note": "whole sequence on its read + write bytes: below 64K tokens the step is bound by kernel "
+                             "launch and dependency latencies, not by one kernel; the dominant kernel by time is named"},
+        "l2_warm": {"ms_per_step": total_warm, "value": total_tokens / (total_warm * 1e-3)},
+        "kernels_ms": kernel_tot, "layers": kinds}))
+
+
 def run_reference(args) -> None:
     """--impl reference: the oracle is the reference arm (no reference implementation exists)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -336,6 +464,9 @@ def main() -> None:
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.workload in LAYER_SEQUENCES:
+        run_layer_sequence(args)
         return
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))      # one rank per GPU; rank 0 prints the line
