@@ -102,8 +102,8 @@ int parked_tiles_per_cta(int max_len, int ctas) {
 }
 
 // The parked kernel's partition mode (several (sequence, head) phases side by side, each on its share of the
-// CTAs, in rounds that fit the grid at one ring of tiles per CTA) can run whenever the longest sequence alone
-// fits the ring and the table of rounds fits its shared memory.
+// CTAs, in waves that fit the grid at one ring of tiles per CTA) can run whenever the longest sequence alone
+// fits the ring and the table of waves fits its shared memory.
 bool partition_ok(const fastkv_shape& s, int ctas, int slots) {
   return static_cast<long long>(s.batch) * s.n_kv_heads <= 512 && parked_tiles_per_cta(s.max_len, ctas) <= slots;
 }
@@ -154,8 +154,8 @@ Layout make_layout(const fastkv_shape& s) {
   // ring (16 tiles per CTA: 303K tokens) the parked kernel with the whole grid on one head at a time; beyond the
   // ring the re-read kernel again.  Batches: see below.  The buffered two-kernel path serves the remaining shapes.
   const int per = parked_tiles_per_cta(s.max_len, kFusedMaxCtas), slots = parked_slots(l.npad);
-  // batches: sequences side by side, in as few rounds as fit the ring (the ring then holds one phase, not two, but
-  // every CTA streams all the time, there are rounds x n_kv_heads phases instead of batch x n_kv_heads, and a
+  // batches: sequences side by side, in as few waves as fit the ring (the ring then holds one phase, not two, but
+  // every CTA streams all the time, there are waves x n_kv_heads phases instead of batch x n_kv_heads, and a
   // statistics exchange involves the CTAs of one sequence only)
   const long long batch_per = (static_cast<long long>(s.total_len) / 128 + kFusedMaxCtas - 1) / kFusedMaxCtas;
   // Partition mode: batches with enough work (sequences x heads exchanges are what it removes: 189 against 266 us

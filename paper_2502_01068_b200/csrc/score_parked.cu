@@ -58,7 +58,7 @@ constexpr int kParkedThreads = 32 * (kCtrlWarps + kPass1Warps + kPass2Warps);   
 constexpr int kMaxStages = 8;
 constexpr int kMaxSlots = 16;
 constexpr int kRefBufs = 4;                    // phases whose references may be waiting for pass 2
-constexpr int kMaxPartUnits = 512;             // (sequence, KV head) pairs a partitioned launch may have (rounds <= units)
+constexpr int kMaxPartUnits = 512;             // (sequence, KV head) pairs a partitioned launch may have (waves <= units)
 // Pass 1 keeps e = exp2(s - ref) with the row's first logit as the reference; the reference only moves
 // when a logit exceeds it by more than this many binary orders of magnitude (e and its row sums stay far
 // inside the fp32 range: e <= 2^64, at most 2^20-odd terms per sum).
@@ -153,15 +153,15 @@ struct PhaseIter {
 
 // Partition mode.  Units of work -- a whole sequence (all its KV heads, one after the other: p.partition == 1,
 // batches) or one KV head of a sequence (p.partition == 2, a single sequence of middling length) -- are taken
-// in rounds of consecutive units; within a round the CTAs of the grid are dealt out to the round's units in
+// in waves of consecutive units; within a wave the CTAs of the grid are dealt out to the wave's units in
 // proportion to their length: this CTA is number `cta` of the `ncta` that share the unit and sees no other
-// unit of the round.  The units of a round are scored side by side, every CTA has tiles in every phase, and a
+// unit of the wave.  The units of a wave are scored side by side, every CTA has tiles in every phase, and a
 // statistics exchange involves only the CTAs of one unit.  That is what batches and shorter sequences want (a
 // grid-wide phase per head would cost sequences x heads exchanges, or leave most CTAs without a tile); a
 // single long sequence is better off with the whole grid on one head at a time and two phases in the ring.
-// One entry per round, worked out once per CTA and kept in shared memory.
+// One entry per wave, worked out once per CTA and kept in shared memory.
 struct PartEntry {
-  int b, g;        // the CTA's unit in this round (g < 0: every head of b in turn); b == kPartIdle: none; kPartEnd: no more rounds
+  int b, g;        // the CTA's unit in this wave (g < 0: every head of b in turn); b == kPartIdle: none; kPartEnd: no more waves
   int cta, ncta;   // its number among the CTAs of that unit, and how many they are
   int per;         // tiles per CTA the deal came out at (at most the ring)
 };
@@ -173,9 +173,9 @@ __device__ __forceinline__ int seq_tiles(const FusedParams& p, int b) {
   return L < p.window ? 0 : (L + kTileKeys - 1) / kTileKeys;       // a sequence shorter than the window has no scores
 }
 
-// The same arithmetic in every CTA.  Rounds are filled greedily: a unit joins the round while the round's
+// The same arithmetic in every CTA.  Waves are filled greedily: a unit joins the wave while the wave's
 // units still fit the grid at `ring` tiles per CTA (one unit always does: the host checked the longest
-// sequence); inside a round the smallest number of tiles per CTA that fits is used.  Run by one thread.
+// sequence); inside a wave the smallest number of tiles per CTA that fits is used.  Run by one thread.
 __device__ void fill_part_table(const FusedParams& p, int cta, int ncta, int ring, PartEntry* tab) {
   const int H = p.partition == 2 ? p.n_kv_heads : 1, units = p.batch * H;
   int u0 = 0, r = 0;
@@ -195,7 +195,7 @@ __device__ void fill_part_table(const FusedParams& p, int cta, int ncta, int rin
       if (n <= ncta) break;
       ++per;
     }
-    PartEntry e = {kPartIdle, 0, 0, 0, per};                          // a CTA left over in this round
+    PartEntry e = {kPartIdle, 0, 0, 0, per};                          // a CTA left over in this wave
     int first = 0;
     for (int u = u0; u < u1; ++u) {
       const int n = (seq_tiles(p, u / H) + per - 1) / per;
@@ -213,8 +213,8 @@ template <bool PART>
 __device__ __forceinline__ bool next_phase(const FusedParams& p, PhaseIter& it, int cta, int ncta, const PartEntry* tab,
                                            PhaseWork& w) {
   int per_fixed = 0;
-  if (PART) {                                              // this CTA's unit of the round: one head, or all heads in turn
-    PartEntry e = tab[it.b];                               // (it.b counts rounds here)
+  if (PART) {                                              // this CTA's unit of the wave: one head, or all heads in turn
+    PartEntry e = tab[it.b];                               // (it.b counts waves here)
     while (e.b == kPartIdle || (e.b >= 0 && it.g >= (e.g < 0 ? p.n_kv_heads : 1))) {
       e = tab[++it.b];
       it.g = 0;
@@ -268,7 +268,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
   float2* norm = warp_stats + 2 * 4 * NPAD;                           // [NPAD] (-row max, 1 / row sum)
   float2* merge_buf = norm + NPAD;                                    // [256] partial merges
   int* row_j = reinterpret_cast<int*>(merge_buf + 2 * kPass2Threads); // [NPAD] window row j = n / G of query row n
-  PartEntry* part_tab = reinterpret_cast<PartEntry*>(row_j + NPAD);   // [rounds + 1], partition mode only
+  PartEntry* part_tab = reinterpret_cast<PartEntry*>(row_j + NPAD);   // [waves + 1], partition mode only
   constexpr int CPW = NPAD / 2;                                       // accumulator columns per pass-1 warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

@@ -129,12 +129,12 @@ def test_parked_kernel_at_the_edge_of_its_ring(debug_hooks):
     assert e.value.status == B.ERR_UNSUPPORTED
 
 
-def test_batch_scored_side_by_side_in_several_rounds(debug_hooks):
+def test_batch_scored_side_by_side_in_several_waves(debug_hooks):
     """A batch on the parked kernel: its sequences are scored side by side, each by its share of the CTAs, in as
-    many rounds as the tensor-memory ring needs (here three: {0, 1}, {2, 3}, {4}); one sequence is much shorter
-    than the others, one round has CTAs left over."""
+    many waves as the tensor-memory ring needs (here three: {0, 1}, {2, 3}, {4}); one sequence is much shorter
+    than the others, one wave has CTAs left over."""
     lens = [150000, 90000, 200000, 4000, 120000]
-    wl = small("rounds", 603, lens, [4000] * 5, [8000, 8000, 8000, 800, 8000], Hq=4, Hkv=1, d=64, hidden=64)
+    wl = small("waves", 603, lens, [4000] * 5, [8000, 8000, 8000, 800, 8000], Hq=4, Hkv=1, d=64, hidden=64)
     x = W.make_layer(wl)
     o = oracle_layer(wl, x)
     check_layer(wl, x, gpu_layer(wl, x), o, what="five sequences, the library's choice")
