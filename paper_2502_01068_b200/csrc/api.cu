@@ -666,7 +666,12 @@ int fastkv_decode_attn(const fastkv_shape* shape, const void* q, const void* k_c
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   const size_t parts = static_cast<size_t>(s.batch) * s.n_kv_heads * kDecodeMaxSplits * G;
   DecodeParams p;
-  p.q = static_cast<const uint16_t*>(q); p.k_cache = k_cache; p.v_cache = v_cache; p.ld_cache = kv->total;
+  CUtensorMap tmap_k, tmap_v;
+  const long long head_stride = static_cast<long long>(kv->total) * s.head_dim;
+  if ((rc = encode_bf16_3d(&tmap_k, k_cache, s.head_dim, s.n_kv_heads, kv->total, head_stride, s.head_dim, 1, 16)) ||
+      (rc = encode_bf16_3d(&tmap_v, v_cache, s.head_dim, s.n_kv_heads, kv->total, head_stride, s.head_dim, 1, 16)))
+    return rc;
+  p.q = static_cast<const uint16_t*>(q); p.ld_cache = kv->total;
   p.cu_k = kv->cu_k; p.k_uniform = kv->k; p.n_q_heads = s.n_q_heads; p.n_kv_heads = s.n_kv_heads; p.group = G;
   const float scale = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / std::sqrt(static_cast<float>(s.head_dim));
   p.scale_log2 = scale * 1.4426950408889634f;
@@ -678,7 +683,7 @@ int fastkv_decode_attn(const fastkv_shape* shape, const void* q, const void* k_c
   cudaError_t e;
   {
     TimedLaunch timed(KID_DECODE, static_cast<cudaStream_t>(stream_));
-    e = launch_decode_attn(p, s.head_dim, s.batch, k_max, static_cast<cudaStream_t>(stream_));
+    e = launch_decode_attn(tmap_k, tmap_v, p, s.head_dim, s.batch, k_max, static_cast<cudaStream_t>(stream_));
   }
   if (e != cudaSuccess) return cuda_fail(e, "decode_attn_kernel launch");
   g_launches += 2;

@@ -9,9 +9,8 @@ constexpr int kDecodeMaxSplits = 64;
 
 struct DecodeParams {
   const uint16_t* q;          // [B][Hq][d] bf16 bits: one new query token per sequence
-  const void* k_cache;        // [Hkv][ld_cache][d] bf16, sequence b at rows cu_k[b] .. (or b * k_uniform ..)
-  const void* v_cache;
-  long long ld_cache;         // kept entries summed over the batch (rows per head)
+  // the caches ([Hkv][ld_cache][d] bf16, sequence b at rows cu_k[b] .. or b * k_uniform ..) come as tensor maps
+  long long ld_cache;         // kept entries summed over the batch (rows per head of the caches)
   const int* cu_k;            // device, may be null (then k_uniform)
   int k_uniform;
   int n_q_heads, n_kv_heads, group;
@@ -24,6 +23,8 @@ struct DecodeParams {
 };
 
 size_t decode_workspace_bytes(int batch, int n_kv_heads, int group, int head_dim);
-cudaError_t launch_decode_attn(DecodeParams& p, int head_dim, int batch, int k_max, cudaStream_t stream);
+// tmap_k / tmap_v: the caches as (column, head, row) tensors, boxes of 64 columns x 1 head x 16 rows, 128-byte swizzle
+cudaError_t launch_decode_attn(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, DecodeParams& p, int head_dim, int batch,
+                               int k_max, cudaStream_t stream);
 
 }  // namespace fastkv

@@ -62,3 +62,20 @@ def test_decode_attention_on_a_compacted_layer_and_with_peaked_softmax():
         got, _ = run_decode(q, g["k_out"], g["v_out"], [128], wl.n_q_heads, wl.n_kv_heads, wl.head_dim, False, scale)
         ref, _ = oracle.decode_attention(q[0], g["k_out"], g["v_out"], scale=None if scale == 0.0 else scale)
         assert np.all(np.abs(got[0] - ref) <= RTOL * np.abs(ref) + ATOL)
+
+
+def test_decode_attention_keeps_sequences_apart_when_a_neighbour_holds_nan():
+    """A chunk of 16 cache rows can straddle two sequences: whatever the neighbour's rows hold (here NaN and
+    infinity in K and V) must not reach this sequence's output."""
+    Hq, Hkv, d, ks = 8, 2, 128, [21, 40, 3]
+    rng = np.random.default_rng(77)
+    q = W.f32_to_bf16_bits(rng.standard_normal((3, Hq, d), dtype=np.float32))
+    kf = rng.standard_normal((Hkv, sum(ks), d), dtype=np.float32)
+    vf = rng.standard_normal((Hkv, sum(ks), d), dtype=np.float32)
+    kf[:, 21:61], vf[:, 21:61] = np.nan, np.inf          # the middle sequence is poisoned
+    kc, vc = W.f32_to_bf16_bits(kf), W.f32_to_bf16_bits(vf)
+    got, got_lse = run_decode(q, kc, vc, ks, Hq, Hkv, d, True)
+    for b, (lo, hi) in ((0, (0, 21)), (2, (61, 64))):
+        ref, ref_lse = oracle.decode_attention(q[b], kc[:, lo:hi], vc[:, lo:hi])
+        assert np.all(np.abs(got[b] - ref) <= RTOL * np.abs(ref) + ATOL)
+        np.testing.assert_allclose(got_lse[b], ref_lse, rtol=1e-5, atol=1e-4)
