@@ -37,7 +37,8 @@ namespace {
 
 constexpr int kBM = 128;                       // queries per CTA
 constexpr int kBN = 128;                       // keys per tile
-constexpr int kAttnThreads = 320;              // producer warp, issuer warp, eight softmax warps
+constexpr int kAttnThreads = 352;              // producer warp, two issuer warps, eight softmax warps
+constexpr int kCtrlWarps = 3;
 constexpr int kSoftmaxWarps = 8;
 constexpr int kChunkBytes = 128 * 128;         // 128 rows x 64 bf16: one swizzled column chunk of a tile
 constexpr float kRescaleSlackLog2 = 8.0f;
@@ -56,6 +57,7 @@ struct AttnBarriers {
   uint64_t s_full[2], s_free[2];
   uint64_t p_full[2], p_free[2];
   uint64_t o_done;
+  uint64_t s_done;              // every S = Q K^T contraction issued has finished
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -82,6 +84,42 @@ __device__ __forceinline__ void tc_mma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a,
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
+}
+
+// Waits of the two control warps.  A control warp waits most of the time, and a polling loop takes issue slots from
+// the two softmax warps that share its scheduler (they handed P over ~0.8 kcycles per tile later than the other six,
+// and the whole pipeline waited for them): the wait is left to the hardware instead, which suspends the thread until
+// the phase completes or the hinted time has passed.  Bounded like every other wait.
+#ifndef FASTKV_PARK_NS
+#define FASTKV_PARK_NS 1000
+#endif
+__device__ __forceinline__ bool mbar_wait_parked(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                 WorkspaceHeader* hdr, int site, long long limit) {
+  const long long t0 = clock64();
+  while (true) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(static_cast<uint32_t>(FASTKV_PARK_NS))
+        : "memory");
+    if (ok) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > limit) {
+      *abort_flag = 1;
+      raise_status(hdr, FASTKV_ERR_DEVICE_TIMEOUT, site);
+      return false;
+    }
+  }
+}
+
+// True in exactly one lane of the (converged) warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -129,6 +167,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     for (int i = 0; i < 2; ++i) { mbar_init(&bars->s_full[i], 1); mbar_init(&bars->s_free[i], kSoftmaxWarps); }
     for (int i = 0; i < 2; ++i) { mbar_init(&bars->p_full[i], kSoftmaxWarps); mbar_init(&bars->p_free[i], 1); }
     mbar_init(&bars->o_done, 1);
+    mbar_init(&bars->s_done, 1);
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -183,58 +222,83 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       }
     }
   } else if (warp == 1) {
-    // ---------------- issuer ----------------
-    if (lane == 0) {
+    // ---------------- issuer of S = Q K^T ----------------
+    // Two issuing warps, on two schedulers: issuing a contraction holds up the other warps of the issuer's
+    // scheduler (with one issuer for both products the two softmax warps next to it handed P over ~0.6 kcycles per
+    // tile after the other six, and every tile waited for them).  Contractions of one thread execute in order; the
+    // two threads' are ordered through the barriers they commit to.
+    // Each issuing warp walks its loop in step, so descriptors, addresses and waits are warp-uniform work; one
+    // elected lane issues each contraction and each commit.
+    {
       constexpr uint32_t idesc_s = umma_idesc_bf16_f32(kBM, kBN);
-      constexpr uint32_t idesc_o = umma_idesc_bf16_f32(kBM, D) | (1u << 16);      // B (V) is MN-major
       const uint32_t q_addr = smem_u32(sQ);
-      bool ok = mbar_wait_bounded(&bars->q_full, 0, abort_flag, p.hdr, SITE_ATTN_Q, limit);
+      bool ok = mbar_wait_parked(&bars->q_full, 0, abort_flag, p.hdr, SITE_ATTN_Q, limit);
+      ok = __all_sync(0xffffffffu, ok);
       int committed = 0;
-      auto second = [&](int t) {                           // O (+)= P_t V_t
-        const int s = t % NS, pb = t & 1;
-        ok = mbar_wait_bounded(&bars->v_full[s], (t / NS) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit) &&
-             mbar_wait_bounded(&bars->p_full[pb], (t >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_P, limit);
-        if (!ok) return;
-        tc_fence_after_sync();
-        // one descriptor per tile; a step further along K only moves its start-address field (units of 16 bytes)
-        const uint64_t b0 = umma_desc_mn_sw128(smem_u32(sV + s * Cfg::kTileBytes), kChunkBytes);
-        const uint32_t a0 = tmem_base + 384 + pb * 64;
-#pragma unroll
-        for (int kk = 0; kk < kBN / 16; ++kk)              // 16 keys = 8 packed columns of P, 2048 bytes of V per step
-          tc_mma_bf16_ts(tmem_base + 256, a0 + kk * 8, b0 + static_cast<uint64_t>(kk * (2048 >> 4)), idesc_o,
-                         (t > 0 || kk > 0) ? 1u : 0u);
-        tc_commit(&bars->v_empty[s]);
-        if (t != p.skip_commit_tile) tc_commit(&bars->p_free[pb]);     // (test hook: a completion that is never signalled)
-        ++committed;
-      };
       for (int j = 0; j < n_tiles && ok; ++j) {
         const int s = j & 1, ks = j % NS;
-        ok = mbar_wait_bounded(&bars->k_full[ks], (j / NS) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit) &&
-             mbar_wait_bounded(&bars->s_free[s], ((j >> 1) & 1) ^ 1, abort_flag, p.hdr, SITE_ATTN_S, limit);
+        ok = mbar_wait_parked(&bars->k_full[ks], (j / NS) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit) &&
+             mbar_wait_parked(&bars->s_free[s], ((j >> 1) & 1) ^ 1, abort_flag, p.hdr, SITE_ATTN_S, limit);
+        ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after_sync();
         const uint64_t a0 = umma_desc_k_sw128(q_addr), b0 = umma_desc_k_sw128(smem_u32(sK + ks * Cfg::kTileBytes));
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {              // 64-element chunk kk / 4, 32 bytes per step inside it
           const uint64_t step = static_cast<uint64_t>(((kk >> 2) * kChunkBytes + (kk & 3) * 32) >> 4);
-          tc_mma_bf16(tmem_base + s * kBN, a0 + step, b0 + step, idesc_s, kk > 0 ? 1u : 0u);
+          if (elect_one()) tc_mma_bf16(tmem_base + s * kBN, a0 + step, b0 + step, idesc_s, kk > 0 ? 1u : 0u);
         }
-        tc_commit(&bars->k_empty[ks]);
-        tc_commit(&bars->s_full[s]);
+        if (elect_one()) {
+          tc_commit(&bars->k_empty[ks]);
+          tc_commit(&bars->s_full[s]);
+        }
         ++committed;
-        if (j >= 1) second(j - 1);
       }
-      if (ok) second(n_tiles - 1);
+      // every contraction this warp issued has finished before tensor memory is released
+      if (committed > 0) {
+        if (elect_one()) tc_commit(&bars->s_done);
+        __syncwarp();
+        mbar_wait_drain(&bars->s_done, 0, p.hdr, SITE_ATTN_DRAIN, limit);
+      }
+    }
+  } else if (warp == 2) {
+    // ---------------- issuer of O (+)= P V ----------------
+    {
+      constexpr uint32_t idesc_o = umma_idesc_bf16_f32(kBM, D) | (1u << 16);      // B (V) is MN-major
+      bool ok = true;
+      int committed = 0;
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int s = t % NS, pb = t & 1;
+        ok = mbar_wait_parked(&bars->v_full[s], (t / NS) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit) &&
+             mbar_wait_parked(&bars->p_full[pb], (t >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_P, limit);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+        // one descriptor per tile; a step further along K only moves its start-address field (units of 16 bytes)
+        const uint64_t b0 = umma_desc_mn_sw128(smem_u32(sV + s * Cfg::kTileBytes), kChunkBytes);
+        const uint32_t a0 = tmem_base + 384 + pb * 64;
+#pragma unroll
+        for (int kk = 0; kk < kBN / 16; ++kk)              // 16 keys = 8 packed columns of P, 2048 bytes of V per step
+          if (elect_one())
+            tc_mma_bf16_ts(tmem_base + 256, a0 + kk * 8, b0 + static_cast<uint64_t>(kk * (2048 >> 4)), idesc_o,
+                           (t > 0 || kk > 0) ? 1u : 0u);
+        if (elect_one()) {
+          tc_commit(&bars->v_empty[s]);
+          if (t != p.skip_commit_tile) tc_commit(&bars->p_free[pb]);   // (test hook: a completion that is never signalled)
+        }
+        ++committed;
+      }
       // every contraction issued has finished before tensor memory is released (and O is complete)
       if (committed > 0) {
-        tc_commit(&bars->o_done);
+        if (elect_one()) tc_commit(&bars->o_done);
+        __syncwarp();
         mbar_wait_drain(&bars->o_done, 0, p.hdr, SITE_ATTN_DRAIN, limit);
       }
     }
   } else {
     // ---------------- softmax: two threads per query row, 64 keys of the tile each ----------------
-    const int gw = warp - 2;
-    const int quarter = warp & 3, half = gw >> 2;         // warps 2..5 and 6..9 cover the four lane quarters once each
+    const int gw = warp - kCtrlWarps;
+    const int quarter = warp & 3, half = gw >> 2;         // warps 3..6 and 7..10 cover the four lane quarters once each
     const int r = quarter * 32 + lane;                    // row of the tile = tensor-memory lane
     const int t = q0 + r;                                 // query position in its sequence
     const int t_eff = min(t, L - 1);                      // rows past the end repeat the last row (never stored)
