@@ -128,6 +128,34 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
   }
 }
 
+// The wait of a control warp (a producer, an issuer).  A control warp waits most of the time, and a polling loop takes
+// issue slots from the compute warps that share its scheduler: the wait is left to the hardware instead, which
+// suspends the thread until the phase completes or the hinted time has passed.  Bounded like every other wait.
+#ifndef FASTKV_PARK_NS
+#define FASTKV_PARK_NS 1000
+#endif
+__device__ __forceinline__ bool mbar_wait_parked(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                 WorkspaceHeader* hdr, int site, long long limit) {
+  const long long t0 = clock64();
+  while (true) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(static_cast<uint32_t>(FASTKV_PARK_NS))
+        : "memory");
+    if (ok) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > limit) {
+      *abort_flag = 1;
+      raise_status(hdr, FASTKV_ERR_DEVICE_TIMEOUT, site);
+      return false;
+    }
+  }
+}
+
 // The wait a role uses for its own copies or contractions still in flight before it leaves: bounded
 // like every other wait, but it does not give up just because the CTA is aborting.
 __device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity, WorkspaceHeader* hdr, int site,
