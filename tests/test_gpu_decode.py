@@ -79,3 +79,36 @@ def test_decode_attention_keeps_sequences_apart_when_a_neighbour_holds_nan():
         ref, ref_lse = oracle.decode_attention(q[b], kc[:, lo:hi], vc[:, lo:hi])
         assert np.all(np.abs(got[b] - ref) <= RTOL * np.abs(ref) + ATOL)
         np.testing.assert_allclose(got_lse[b], ref_lse, rtol=1e-5, atol=1e-4)
+
+
+@pytest.mark.parametrize("seed", [31, 32, 33])
+def test_decode_attention_on_random_shapes(seed):
+    """Seeded random caches: KV heads, group size (1..8, odd ones included), head dimension, batch size and kept
+    entries per sequence (empty caches, caches shorter than one 16-entry chunk, caches of thousands of entries), a
+    random softmax scale; every sequence against its own oracle run."""
+    rng = np.random.default_rng(seed)
+    for it in range(6):
+        Hkv = int(rng.choice([1, 2, 3, 8])); G = int(rng.integers(1, 9)); d = int(rng.choice([64, 128]))
+        Bn = int(rng.integers(1, 6))
+        ks = [int(rng.choice([0, 1, 15, 16, 17, int(rng.integers(18, 400)), int(rng.integers(400, 6000))])) for _ in range(Bn)]
+        if sum(ks) == 0:
+            ks[0] = 33
+        if Bn == 1 or len(set(ks)) == 1:
+            ks = [max(ks[0], 1)] * Bn                      # the uniform form of the budget
+        scale = float(rng.choice([0.0, 0.05, 0.5]))
+        Hq, tot = Hkv * G, sum(ks)
+        q = W.f32_to_bf16_bits(rng.standard_normal((Bn, Hq, d), dtype=np.float32))
+        kc = W.f32_to_bf16_bits(rng.standard_normal((Hkv, tot, d), dtype=np.float32))
+        vc = W.f32_to_bf16_bits(rng.standard_normal((Hkv, tot, d), dtype=np.float32))
+        ragged = len(set(ks)) > 1
+        got, got_lse = run_decode(q, kc, vc, ks, Hq, Hkv, d, ragged, scale)
+        cu = np.concatenate([[0], np.cumsum(ks)])
+        for b in range(Bn):
+            if ks[b] == 0:
+                assert np.all(got[b] == 0.0), (seed, it, b)   # an empty cache: the output is defined as zero
+                continue
+            ref, ref_lse = oracle.decode_attention(q[b], kc[:, cu[b]:cu[b + 1]], vc[:, cu[b]:cu[b + 1]],
+                                                   scale=None if scale == 0.0 else scale)
+            err = np.abs(got[b] - ref)
+            assert np.all(err <= RTOL * np.abs(ref) + ATOL), (seed, it, b, Hkv, G, d, ks, float(err.max()))
+            np.testing.assert_allclose(got_lse[b], ref_lse, rtol=1e-5, atol=1e-4)
