@@ -681,12 +681,13 @@ int fastkv_decode_attn(const fastkv_shape* shape, const void* q, const void* k_c
   p.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
   const int k_max = kv->cu_k ? (kv->total < s.max_len ? kv->total : s.max_len) : kv->k;
   cudaError_t e;
+  int launched = 0;
   {
     TimedLaunch timed(KID_DECODE, static_cast<cudaStream_t>(stream_));
-    e = launch_decode_attn(tmap_k, tmap_v, p, s.head_dim, s.batch, k_max, static_cast<cudaStream_t>(stream_));
+    e = launch_decode_attn(tmap_k, tmap_v, p, s.head_dim, s.batch, k_max, static_cast<cudaStream_t>(stream_), &launched);
   }
+  g_launches += launched;
   if (e != cudaSuccess) return cuda_fail(e, "decode_attn_kernel launch");
-  g_launches += 2;
   return FASTKV_OK;
 }
 

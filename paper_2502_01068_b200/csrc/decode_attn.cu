@@ -255,8 +255,15 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       L = fmaf(ml.y, f, L);
       acc = fmaf(mo[(w * kDecHeads + h) * D + col], f, acc);
     }
-    if (col == 0) p.part_ml[part + h] = make_float2(M, L);
-    p.part_o[(part + h) * D + col] = acc;
+    if (n_splits == 1) {
+      // the only split of this (sequence, KV head): the result is final, no merge kernel follows
+      const size_t row = static_cast<size_t>(b) * p.n_q_heads + g * G + h;
+      p.out[row * D + col] = L > 0.0f ? acc / L : 0.0f;
+      if (p.lse != nullptr && col == 0) p.lse[row] = (M + log2f(L)) * 0.6931471805599453f;
+    } else {
+      if (col == 0) p.part_ml[part + h] = make_float2(M, L);
+      p.part_o[(part + h) * D + col] = acc;
+    }
   }
 }
 
@@ -298,7 +305,7 @@ size_t decode_workspace_bytes(int batch, int n_kv_heads, int group, int head_dim
 
 template <int D>
 static cudaError_t launch_decode_d(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, int batch, int k_max,
-                                   cudaStream_t stream) {
+                                   cudaStream_t stream, int* launches) {
   constexpr int kSmem = DecCfg<D>::kSmem;
   // launch attributes and occupancy are per device: cached by device ordinal
   static PerDeviceOnce configured;
@@ -328,6 +335,9 @@ static cudaError_t launch_decode_d(const CUtensorMap& tk, const CUtensorMap& tv,
   decode_attn_kernel<D><<<dim3(splits, p.n_kv_heads, batch), kDecThreads, kSmem, stream>>>(tk, tv, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
+  *launches = 1;
+  if (splits == 1) return cudaSuccess;          // the split kernel wrote the output itself
+  *launches = 2;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(p.n_q_heads, batch);
   cfg.blockDim = dim3(D);
@@ -340,9 +350,10 @@ static cudaError_t launch_decode_d(const CUtensorMap& tk, const CUtensorMap& tv,
 }
 
 cudaError_t launch_decode_attn(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, DecodeParams& p, int head_dim, int batch,
-                               int k_max, cudaStream_t stream) {
-  if (head_dim == 128) return launch_decode_d<128>(tmap_k, tmap_v, p, batch, k_max, stream);
-  if (head_dim == 64) return launch_decode_d<64>(tmap_k, tmap_v, p, batch, k_max, stream);
+                               int k_max, cudaStream_t stream, int* launches) {
+  *launches = 0;
+  if (head_dim == 128) return launch_decode_d<128>(tmap_k, tmap_v, p, batch, k_max, stream, launches);
+  if (head_dim == 64) return launch_decode_d<64>(tmap_k, tmap_v, p, batch, k_max, stream, launches);
   return cudaErrorInvalidValue;
 }
 

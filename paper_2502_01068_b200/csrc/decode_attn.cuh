@@ -24,7 +24,8 @@ struct DecodeParams {
 
 size_t decode_workspace_bytes(int batch, int n_kv_heads, int group, int head_dim);
 // tmap_k / tmap_v: the caches as (column, head, row) tensors, boxes of 64 columns x 1 head x 16 rows, 128-byte swizzle
+// *launches: kernels launched (1 when every (sequence, KV head) has a single split: no merge kernel then)
 cudaError_t launch_decode_attn(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, DecodeParams& p, int head_dim, int batch,
-                               int k_max, cudaStream_t stream);
+                               int k_max, cudaStream_t stream, int* launches);
 
 }  // namespace fastkv
