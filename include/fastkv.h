@@ -263,9 +263,9 @@ int fastkv_score_static_status(void* stream, int32_t* status, int32_t* site);
  *   "extra_publications"  the scoring kernels' second pass waits for this many publications of
  *                         softmax statistics beyond those that will arrive; with a short wait limit
  *                         this makes a bounded wait run out without any fault (timeout test)
- *   "prefill_skip_commit" n > 0: the prefill attention's issuer withholds the signal that P of key tile
- *                         n - 1 was consumed; with a short wait limit the softmax warps' bounded wait
- *                         runs out without any fault (timeout test); 0: off
+ *   "prefill_skip_commit" n > 0: the prefill attention's issuer withholds the signal that S of key tile
+ *                         n - 1 is ready (first query tile of every CTA); with a short wait limit the
+ *                         softmax warps' bounded wait runs out without any fault (timeout test); 0: off
  *   "time_kernels"        1: record a pair of CUDA events around every kernel the library launches
  *                         (this creates events, and an event between two kernels keeps the second
  *                         from starting under the first one's tail); read with

@@ -46,7 +46,7 @@ struct DebugConfig {
   long long wait_limit_cycles = 0;  // 0 = the default of about a second
   int extra_publications = 0;       // pass 2 waits for publications that never come (timeout test)
   int score_partition = 0;          // parked kernel's partition mode: 0 = by shape, 1 = never, 2 = whenever it can run
-  int prefill_skip_commit = 0;      // prefill attention: n > 0: key tile n - 1's "P consumed" signal is withheld (timeout test)
+  int prefill_skip_commit = 0;      // prefill attention: n > 0: key tile n - 1's "S ready" signal is withheld (timeout test)
 };
 DebugConfig g_debug;
 

@@ -35,11 +35,11 @@ namespace fastkv {
 
 namespace {
 
-constexpr int kBM = 128;                       // queries per CTA
+constexpr int kBM = 128;                       // queries per query tile; a CTA has two of them
 constexpr int kBN = 128;                       // keys per tile
-constexpr int kAttnThreads = 352;              // producer warp, two issuer warps, eight softmax warps
-constexpr int kCtrlWarps = 3;
-constexpr int kSoftmaxWarps = 8;
+constexpr int kCtrlWarps = 3;                  // producer, issuer of query tile A, issuer of query tile B
+constexpr int kSoftmaxWarps = 8;               // per query tile
+constexpr int kAttnThreads = (kCtrlWarps + 2 * kSoftmaxWarps) * 32;
 constexpr int kChunkBytes = 128 * 128;         // 128 rows x 64 bf16: one swizzled column chunk of a tile
 constexpr float kRescaleSlackLog2 = 8.0f;
 
@@ -47,17 +47,18 @@ template <int D>
 struct AttnCfg {
   static constexpr int KH = D / 64;
   static constexpr int kTileBytes = KH * kChunkBytes;     // Q, K or V tile
-  static constexpr int kKvStages = 3;
-  static constexpr int kSmemBytes = (1 + 2 * kKvStages) * kTileBytes + 256 + 2 * 2 * kBM * 4;
+  static constexpr int kKvStages = 2;
+  // two Q tiles, the K and V rings, the barriers, what the two halves of a row exchange ([tile][2][2][128] floats)
+  static constexpr int kSmemBytes = (2 + 2 * kKvStages) * kTileBytes + 256 + 2 * 2 * 2 * kBM * 4;
 };
 
 struct AttnBarriers {
   uint64_t q_full;
-  uint64_t k_full[3], k_empty[3], v_full[3], v_empty[3];
-  uint64_t s_full[2], s_free[2];
-  uint64_t p_full[2], p_free[2];
-  uint64_t o_done;
-  uint64_t s_done;              // every S = Q K^T contraction issued has finished
+  uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // empty: both issuers are done with the stage
+  uint64_t s_full[2];           // per query tile: S = Q K^T of the current key tile is in tensor memory
+  uint64_t p_full[2];           // per query tile: every softmax warp has stored its part of P
+  uint64_t o_done[2];           // per query tile: every contraction its issuer started has finished
+  uint64_t turn[2];             // turn[x]: the other tile's issuer has issued the block that goes before x's next one
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -107,38 +108,43 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                     const __grid_constant__ CUtensorMap tmap_v, const PrefillParams p) {
   using Cfg = AttnCfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];       // the tiles need 1024-byte alignment (128-byte swizzle atoms)
-  uint8_t* sQ = smem;
+  uint8_t* sQ = smem;                                     // two query tiles
   constexpr int NS = Cfg::kKvStages;
-  uint8_t* sK = sQ + Cfg::kTileBytes;                     // NS stages
+  uint8_t* sK = sQ + 2 * Cfg::kTileBytes;                 // NS stages
   uint8_t* sV = sK + NS * Cfg::kTileBytes;                // NS stages
   AttnBarriers* bars = reinterpret_cast<AttnBarriers*>(sV + NS * Cfg::kTileBytes);
-  float* xch = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 256);   // [2][2][128]: what the two halves of a row exchange
+  float* xch_all = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 256);   // [tile][2][2][128]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.z, h = blockIdx.y, g = h / p.group;
   const int row0 = p.cu_seqlens ? p.cu_seqlens[b] : 0;
   const int L = p.cu_seqlens ? p.cu_seqlens[b + 1] - row0 : p.total_len;
-  const int n_qtiles = (L + kBM - 1) / kBM;
-  const int qi = n_qtiles - 1 - static_cast<int>(blockIdx.x);      // the longest rows first
-  if (qi < 0) return;                                              // (uniform per CTA, before any barrier)
+  const int n_pairs = (L + 2 * kBM - 1) / (2 * kBM);
+  const int qp = n_pairs - 1 - static_cast<int>(blockIdx.x);       // the longest rows first
+  if (qp < 0) return;                                              // (uniform per CTA, before any barrier)
   if (smem_u32(smem) & 1023u) {                                    // never seen; would garble every tile
     if (threadIdx.x == 0) raise_status(p.hdr, FASTKV_ERR_UNSUPPORTED, SITE_ATTN_Q);
     return;
   }
-  const int q0 = qi * kBM;
-  const int n_tiles = qi + 1;                                      // key tiles 0 .. qi (causal)
+  const int q0 = qp * 2 * kBM;
+  const bool b_active = q0 + kBM < L;                              // the sequence may end inside query tile A
+  // key tiles of each query tile (causal): A sees 0 .. 2 qp, B one more; the rings carry the longer list
+  const int n_key_a = 2 * qp + 1, n_key_b = b_active ? 2 * qp + 2 : 0;
+  const int n_tiles = b_active ? n_key_b : n_key_a;
   const long long limit = p.wait_limit;
 
   if (threadIdx.x == 0) {
     mbar_init(&bars->q_full, 1);
     for (int i = 0; i < NS; ++i) {
-      mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], 1);
-      mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], 1);
+      mbar_init(&bars->k_full[i], 1); mbar_init(&bars->k_empty[i], 2);
+      mbar_init(&bars->v_full[i], 1); mbar_init(&bars->v_empty[i], 2);
     }
-    for (int i = 0; i < 2; ++i) { mbar_init(&bars->s_full[i], 1); mbar_init(&bars->s_free[i], kSoftmaxWarps); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&bars->p_full[i], kSoftmaxWarps); mbar_init(&bars->p_free[i], 1); }
-    mbar_init(&bars->o_done, 1);
-    mbar_init(&bars->s_done, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bars->s_full[i], 1);
+      mbar_init(&bars->p_full[i], kSoftmaxWarps);
+      mbar_init(&bars->o_done[i], 1);
+      mbar_init(&bars->turn[i], 1);
+    }
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -162,20 +168,22 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     // ---------------- producer ----------------
     if (lane == 0) {
       const uint64_t pol_q = l2_policy_evict_first();      // a Q tile is read by one CTA
-      const uint64_t pol_kv = l2_policy_evict_last();      // K / V tiles are read by every later query tile
-      mbar_arrive_expect_tx(&bars->q_full, Cfg::kTileBytes);
-      for (int c = 0; c < Cfg::KH; ++c) tma_load_3d(sQ + c * kChunkBytes, &tmap_q, &bars->q_full, c * 64, h, row0 + q0, pol_q);
+      const uint64_t pol_kv = l2_policy_evict_last();      // K / V tiles are read by every later pair of query tiles
+      mbar_arrive_expect_tx(&bars->q_full, (b_active ? 2 : 1) * Cfg::kTileBytes);
+      for (int x = 0; x < (b_active ? 2 : 1); ++x)
+        for (int c = 0; c < Cfg::KH; ++c)
+          tma_load_3d(sQ + x * Cfg::kTileBytes + c * kChunkBytes, &tmap_q, &bars->q_full, c * 64, h, row0 + q0 + x * kBM, pol_q);
       bool ok = true;
       int issued = 0;
       for (int j = 0; j < n_tiles && ok; ++j) {
         const int s = j % NS;
         const uint32_t par = (j / NS) & 1;
-        ok = mbar_wait_bounded(&bars->k_empty[s], par ^ 1, abort_flag, p.hdr, SITE_ATTN_RING, limit);
+        ok = mbar_wait_parked(&bars->k_empty[s], par ^ 1, abort_flag, p.hdr, SITE_ATTN_RING, limit);
         if (!ok) break;
         mbar_arrive_expect_tx(&bars->k_full[s], Cfg::kTileBytes);
         for (int c = 0; c < Cfg::KH; ++c)
           tma_load_3d(sK + s * Cfg::kTileBytes + c * kChunkBytes, &tmap_k, &bars->k_full[s], c * 64, g, row0 + j * kBN, pol_kv);
-        ok = mbar_wait_bounded(&bars->v_empty[s], par ^ 1, abort_flag, p.hdr, SITE_ATTN_RING, limit);
+        ok = mbar_wait_parked(&bars->v_empty[s], par ^ 1, abort_flag, p.hdr, SITE_ATTN_RING, limit);
         if (!ok) {                                          // K of this tile is in flight, V is not
           mbar_wait_drain(&bars->k_full[s], par, p.hdr, SITE_ATTN_DRAIN, limit);
           break;
@@ -192,124 +200,147 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         mbar_wait_drain(&bars->v_full[j % NS], (j / NS) & 1, p.hdr, SITE_ATTN_DRAIN, limit);
       }
     }
-  } else if (warp == 1) {
-    // ---------------- issuer of S = Q K^T ----------------
-    // Two issuing warps, on two schedulers: issuing a contraction holds up the other warps of the issuer's
-    // scheduler (with one issuer for both products the two softmax warps next to it handed P over ~0.6 kcycles per
-    // tile after the other six, and every tile waited for them).  Contractions of one thread execute in order; the
-    // two threads' are ordered through the barriers they commit to.
-    // Each issuing warp walks its loop in step, so descriptors, addresses and waits are warp-uniform work; one
-    // elected lane issues each contraction and each commit.
-    {
-      constexpr uint32_t idesc_s = umma_idesc_bf16_f32(kBM, kBN);
-      const uint32_t q_addr = smem_u32(sQ);
-      bool ok = mbar_wait_parked(&bars->q_full, 0, abort_flag, p.hdr, SITE_ATTN_Q, limit);
+  } else if (warp < kCtrlWarps) {
+    // ---------------- issuer of one query tile ----------------
+    // A query tile's contractions come from one thread and therefore execute in the order S(0), O += P V (0), S(1),
+    // O += P V (1), ...: S of the next key tile overwrites the tile's S / P columns only after the contraction that
+    // read P from them, and the softmax of key tile j finds O complete up to j - 1, with no barrier for either.
+    // The two tiles' issuers sit on two warp schedulers (issuing a contraction holds up the other warps of the
+    // issuer's scheduler); each walks its loop as a whole warp, one elected lane issues.
+    const int x = warp - 1;
+    const int nk = x == 0 ? n_key_a : n_key_b;
+    constexpr uint32_t idesc_s = umma_idesc_bf16_f32(kBM, kBN);
+    constexpr uint32_t idesc_o = umma_idesc_bf16_f32(kBM, D) | (1u << 16);      // B (V) is MN-major
+    const uint32_t q_addr = smem_u32(sQ + x * Cfg::kTileBytes);
+    const uint32_t s_tmem = tmem_base + x * kBN, o_tmem = tmem_base + 256 + x * D;
+    bool ok = true;
+    int committed = 0;
+    auto first = [&](int j) {                              // S = Q K_j^T
+      const int ks = j % NS;
+      ok = mbar_wait_parked(&bars->k_full[ks], (j / NS) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit);
       ok = __all_sync(0xffffffffu, ok);
-      int committed = 0;
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int s = j & 1, ks = j % NS;
-        ok = mbar_wait_parked(&bars->k_full[ks], (j / NS) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit) &&
-             mbar_wait_parked(&bars->s_free[s], ((j >> 1) & 1) ^ 1, abort_flag, p.hdr, SITE_ATTN_S, limit);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        tc_fence_after_sync();
-        const uint64_t a0 = umma_desc_k_sw128(q_addr), b0 = umma_desc_k_sw128(smem_u32(sK + ks * Cfg::kTileBytes));
+      if (!ok) return;
+      tc_fence_after_sync();
+      const uint64_t a0 = umma_desc_k_sw128(q_addr), b0 = umma_desc_k_sw128(smem_u32(sK + ks * Cfg::kTileBytes));
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {              // 64-element chunk kk / 4, 32 bytes per step inside it
-          const uint64_t step = static_cast<uint64_t>(((kk >> 2) * kChunkBytes + (kk & 3) * 32) >> 4);
-          if (elect_one()) tc_mma_bf16(tmem_base + s * kBN, a0 + step, b0 + step, idesc_s, kk > 0 ? 1u : 0u);
-        }
-        if (elect_one()) {
-          tc_commit(&bars->k_empty[ks]);
-          tc_commit(&bars->s_full[s]);
-        }
-        ++committed;
+      for (int kk = 0; kk < D / 16; ++kk) {                // 64-element chunk kk / 4, 32 bytes per step inside it
+        const uint64_t step = static_cast<uint64_t>(((kk >> 2) * kChunkBytes + (kk & 3) * 32) >> 4);
+        if (elect_one()) tc_mma_bf16(s_tmem, a0 + step, b0 + step, idesc_s, kk > 0 ? 1u : 0u);
       }
-      // every contraction this warp issued has finished before tensor memory is released
-      if (committed > 0) {
-        if (elect_one()) tc_commit(&bars->s_done);
-        __syncwarp();
-        mbar_wait_drain(&bars->s_done, 0, p.hdr, SITE_ATTN_DRAIN, limit);
+      if (elect_one()) {
+        tc_commit(&bars->k_empty[ks]);
+        if (!(x == 0 && j == p.skip_commit_tile)) tc_commit(&bars->s_full[x]);   // (test hook: a completion that is never signalled)
       }
+      ++committed;
+    };
+    auto second = [&](int j) {                             // O (+)= P_j V_j
+      const int s = j % NS;
+      // one descriptor per tile; a step further along K only moves its start-address field (units of 16 bytes).
+      // P: each half of a row keeps its 64 keys, packed, in the first 32 of its own 64 S columns
+      const uint64_t b0 = umma_desc_mn_sw128(smem_u32(sV + s * Cfg::kTileBytes), kChunkBytes);
+#pragma unroll
+      for (int kk = 0; kk < kBN / 16; ++kk)                // 16 keys = 8 packed columns of P, 2048 bytes of V per step
+        if (elect_one())
+          tc_mma_bf16_ts(o_tmem, s_tmem + (kk >> 2) * 64 + (kk & 3) * 8, b0 + static_cast<uint64_t>(kk * (2048 >> 4)), idesc_o,
+                         (j > 0 || kk > 0) ? 1u : 0u);
+      if (elect_one()) tc_commit(&bars->v_empty[s]);
+      ++committed;
+    };
+    if (nk > 0) {
+      ok = mbar_wait_parked(&bars->q_full, 0, abort_flag, p.hdr, SITE_ATTN_Q, limit);
+      ok = __all_sync(0xffffffffu, ok);
     }
-  } else if (warp == 2) {
-    // ---------------- issuer of O (+)= P V ----------------
-    {
-      constexpr uint32_t idesc_o = umma_idesc_bf16_f32(kBM, D) | (1u << 16);      // B (V) is MN-major
-      bool ok = true;
-      int committed = 0;
-      for (int t = 0; t < n_tiles && ok; ++t) {
-        const int s = t % NS, pb = t & 1;
-        ok = mbar_wait_parked(&bars->v_full[s], (t / NS) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit) &&
-             mbar_wait_parked(&bars->p_full[pb], (t >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_P, limit);
+    // Block jb of a tile = [O += P V of key tile jb - 1] [S of key tile jb].  The two tiles' blocks alternate on the
+    // tensor cores -- A(0) B(0) A(1) B(1) ... -- which keeps the two softmaxes half a period apart: one tile's
+    // exponentials run under the other's contractions (left alone, the two tiles fall into step, want the tensor
+    // cores at the same time and the special-function unit at the same time, and each waits while the other works).
+    int jb = 0;
+    for (; nk > 0 && jb <= nk && ok; ++jb) {
+      if (jb > 0) {
+        ok = mbar_wait_parked(&bars->v_full[(jb - 1) % NS], ((jb - 1) / NS) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit) &&
+             mbar_wait_parked(&bars->p_full[x], (jb - 1) & 1, abort_flag, p.hdr, SITE_ATTN_P, limit);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        tc_fence_after_sync();
-        // one descriptor per tile; a step further along K only moves its start-address field (units of 16 bytes)
-        const uint64_t b0 = umma_desc_mn_sw128(smem_u32(sV + s * Cfg::kTileBytes), kChunkBytes);
-        const uint32_t a0 = tmem_base + 384 + pb * 64;
-#pragma unroll
-        for (int kk = 0; kk < kBN / 16; ++kk)              // 16 keys = 8 packed columns of P, 2048 bytes of V per step
-          if (elect_one())
-            tc_mma_bf16_ts(tmem_base + 256, a0 + kk * 8, b0 + static_cast<uint64_t>(kk * (2048 >> 4)), idesc_o,
-                           (t > 0 || kk > 0) ? 1u : 0u);
-        if (elect_one()) {
-          tc_commit(&bars->v_empty[s]);
-          if (t != p.skip_commit_tile) tc_commit(&bars->p_free[pb]);   // (test hook: a completion that is never signalled)
-        }
-        ++committed;
       }
-      // every contraction issued has finished before tensor memory is released (and O is complete)
-      if (committed > 0) {
-        if (elect_one()) tc_commit(&bars->o_done);
-        __syncwarp();
-        mbar_wait_drain(&bars->o_done, 0, p.hdr, SITE_ATTN_DRAIN, limit);
+      if (b_active) {
+        if (x == 0 && jb >= 1) ok = mbar_wait_parked(&bars->turn[0], (jb - 1) & 1, abort_flag, p.hdr, SITE_ATTN_S, limit);
+        if (x == 1 && jb <= n_key_a) ok = mbar_wait_parked(&bars->turn[1], jb & 1, abort_flag, p.hdr, SITE_ATTN_S, limit);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
       }
+      tc_fence_after_sync();
+      if (jb > 0) second(jb - 1);
+      if (jb < nk) first(jb);
+      if (b_active && elect_one()) mbar_arrive(&bars->turn[x ^ 1]);
+    }
+    const bool all_issued = ok && jb > nk;
+    // key tiles this query tile does not use (A has one fewer than B; a tile past the end of the sequence uses none):
+    // the stage still counts two releases
+    for (int jj = (nk == 0 || all_issued) ? nk : n_tiles; jj < n_tiles; ++jj) {
+      const int s = jj % NS;
+      bool fine = mbar_wait_parked(&bars->k_full[s], (jj / NS) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit);
+      fine = __all_sync(0xffffffffu, fine);
+      if (!fine) break;
+      if (lane == 0) mbar_arrive(&bars->k_empty[s]);
+      fine = mbar_wait_parked(&bars->v_full[s], (jj / NS) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit);
+      fine = __all_sync(0xffffffffu, fine);
+      if (!fine) break;
+      if (lane == 0) mbar_arrive(&bars->v_empty[s]);
+    }
+    // every contraction issued has finished before tensor memory is released (and O is complete)
+    if (committed > 0) {
+      if (elect_one()) tc_commit(&bars->o_done[x]);
+      __syncwarp();
+      mbar_wait_drain(&bars->o_done[x], 0, p.hdr, SITE_ATTN_DRAIN, limit);
     }
   } else {
-    // ---------------- softmax: two threads per query row, 64 keys of the tile each ----------------
+    // ---------------- softmax: eight warps per query tile, two threads per query row, 64 keys of the tile each ----------------
     const int gw = warp - kCtrlWarps;
-    const int quarter = warp & 3, half = gw >> 2;         // warps 3..6 and 7..10 cover the four lane quarters once each
+    const int x = gw >> 3, g8 = gw & 7;                   // query tile; warp of the tile
+    const int quarter = warp & 3, half = g8 >> 2;         // a tile's warps cover the four lane quarters twice
+    const int nk = x == 0 ? n_key_a : n_key_b;
     const int r = quarter * 32 + lane;                    // row of the tile = tensor-memory lane
-    const int t = q0 + r;                                 // query position in its sequence
+    const int t = q0 + x * kBM + r;                       // query position in its sequence
     const int t_eff = min(t, L - 1);                      // rows past the end repeat the last row (never stored)
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    const uint32_t s_addr = lane_addr + x * kBN + half * 64;          // this thread's 64 S columns; P goes into the first 32
+    const uint32_t o_addr = lane_addr + 256 + x * D + half * (D / 2); // this thread's D / 2 columns of O
+    float* const xch = xch_all + x * (2 * 2 * kBM);
     const int jw = t - (L - p.window);                    // window row index, if 0 <= jw < w
     const bool is_window = p.wlog != nullptr && jw >= 0 && t < L;
     float* const wlog_row = is_window ? p.wlog + (static_cast<size_t>(h) * p.window + jw) * p.ld_w + row0 : nullptr;
     constexpr int HN = kBN / 2;                           // keys per thread and tile
-    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + (gw & 3)) : "memory"); };
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + x * 4 + (g8 & 3)) : "memory"); };
     float m_ref = -INFINITY, l = 0.0f;                    // the reference is the same in both threads of a row; l is this half's
     bool ok = true;
     // Both warps of a pair walk every tile and meet at the pair's barrier once per tile whatever happens: a
     // warp whose wait gave up skips the work of the tile, never the barrier.
-    for (int j = 0; j < n_tiles; ++j) {
+    for (int j = 0; j < nk; ++j) {
       const int s = j & 1;
-      if (ok) ok = mbar_wait_bounded(&bars->s_full[s], (j >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_SFULL, limit);
+      if (ok) ok = mbar_wait_bounded(&bars->s_full[x], j & 1, abort_flag, p.hdr, SITE_ATTN_SFULL, limit);
       ok = __all_sync(0xffffffffu, ok);
       const int key0 = j * kBN + half * HN;
       const bool diagonal = key0 + HN - 1 > t_eff;        // some keys of this half are not visible to this row
-      float v[HN];
       float half_max = -INFINITY;
       if (ok) {
         tc_fence_after_sync();
-        // this half of the row in registers; the S buffer goes back to the issuer at once
+        // first reading of this half of the row: its maximum (the row stays in tensor memory: a thread holds 32 of
+        // its 64 logits at a time)
 #pragma unroll
-        for (int c = 0; c < HN / 32; ++c)
-          tmem_ld_32x32(lane_addr + s * kBN + half * HN + c * 32, *reinterpret_cast<float (*)[32]>(&v[c * 32]));
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bars->s_free[s]);
-        if (diagonal) {
+        for (int c = 0; c < HN / 32; ++c) {
+          float v[32];
+          tmem_ld_32x32(s_addr + c * 32, v);
+          if (diagonal) {
 #pragma unroll
-          for (int x = 0; x < HN; ++x) v[x] = key0 + x <= t_eff ? v[x] : -INFINITY;
+            for (int i = 0; i < 32; ++i) v[i] = key0 + c * 32 + i <= t_eff ? v[i] : -INFINITY;
+          }
+          float mx[4] = {v[0], v[1], v[2], v[3]};
+#pragma unroll
+          for (int i = 4; i < 32; i += 4) {
+            mx[0] = fmaxf(mx[0], v[i]); mx[1] = fmaxf(mx[1], v[i + 1]); mx[2] = fmaxf(mx[2], v[i + 2]); mx[3] = fmaxf(mx[3], v[i + 3]);
+          }
+          half_max = fmaxf(half_max, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])));
         }
-        float mx[4] = {v[0], v[1], v[2], v[3]};
-#pragma unroll
-        for (int x = 4; x < HN; x += 4) {
-          mx[0] = fmaxf(mx[0], v[x]); mx[1] = fmaxf(mx[1], v[x + 1]); mx[2] = fmaxf(mx[2], v[x + 2]); mx[3] = fmaxf(mx[3], v[x + 3]);
-        }
-        half_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
       }
       xch[(s * 2 + half) * kBM + r] = half_max;
       pair_sync();
@@ -320,91 +351,92 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       const float alpha = move ? ex2(m_ref - tile_max) : 1.0f;     // 0 at the first tile
       if (move) { m_ref = tile_max; l *= alpha; }
       if (j >= 1 && __any_sync(0xffffffffu, move)) {
-        // O is rescaled (each half its own columns) once the second contraction of the tile before has been added to it
-        ok = mbar_wait_bounded(&bars->p_free[(j - 1) & 1], ((j - 1) >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_PFREE, limit);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) continue;
-        tc_fence_after_sync();
+        // O is rescaled, each half its own columns.  It is complete up to key tile j - 1: the contraction that
+        // produced this S was issued after the one that added tile j - 1, by the same thread.
 #pragma unroll
         for (int c = 0; c < D / 64; ++c) {
           float o[32];
-          const uint32_t addr = lane_addr + 256 + half * (D / 2) + c * 32;
-          tmem_ld_32x32(addr, o);
+          tmem_ld_32x32(o_addr + c * 32, o);
 #pragma unroll
-          for (int x = 0; x < 32; ++x) o[x] *= alpha;
-          tmem_st_32x32(addr, o);
+          for (int i = 0; i < 32; ++i) o[i] *= alpha;
+          tmem_st_32x32(o_addr + c * 32, o);
         }
         tmem_wait_st();
       }
-      if (is_window) {                                     // by-product: this row's logits (log2 units), masked = -inf
-        float* const dst = wlog_row + key0;
-        if (key0 + HN <= L && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
-#pragma unroll
-          for (int x = 0; x < HN; x += 4)
-            *reinterpret_cast<float4*>(dst + x) = make_float4(v[x] * p.scale_log2, v[x + 1] * p.scale_log2,
-                                                              v[x + 2] * p.scale_log2, v[x + 3] * p.scale_log2);
-        } else {
-#pragma unroll
-          for (int x = 0; x < HN; ++x)
-            if (key0 + x < L) dst[x] = v[x] * p.scale_log2;
-        }
-      }
-      // this P buffer was last read by the second contraction of tile j - 2
-      if (j >= 2) {
-        ok = mbar_wait_bounded(&bars->p_free[s], ((j - 2) >> 1) & 1, abort_flag, p.hdr, SITE_ATTN_PFREE, limit);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) continue;
-      }
-      // p = exp2(s * scale - ref), the row sum, P in bf16 for the second contraction: two keys per 32-bit column
-      // of tensor memory, this half's 64 keys in 32 columns of the tile's P buffer
+      // second reading: p = exp2(s * scale - ref), the row sum, P in bf16 for the second contraction: two keys per
+      // 32-bit column, this thread's 64 keys in the first 32 of its own 64 S columns (columns it has read already)
       const float neg_ref = -m_ref;
       float ls[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-      float packed[HN / 2];
 #pragma unroll
-      for (int x = 0; x < HN; x += 2) {
-        const float e0 = ex2(fmaf(v[x], p.scale_log2, neg_ref));      // exp2(-inf) = 0 for a masked key
-        const float e1 = ex2(fmaf(v[x + 1], p.scale_log2, neg_ref));
-        ls[x & 2] += e0;
-        ls[(x & 2) + 1] += e1;
-        packed[x / 2] = __uint_as_float(pack_bf16(e0, e1));
+      for (int c = 0; c < HN / 32; ++c) {
+        float v[32];
+        tmem_ld_32x32(s_addr + c * 32, v);
+        if (diagonal) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = key0 + c * 32 + i <= t_eff ? v[i] : -INFINITY;
+        }
+        if (is_window) {                                   // by-product: this row's logits (log2 units), masked = -inf
+          float* const dst = wlog_row + key0 + c * 32;
+          if (key0 + c * 32 + 32 <= L && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              *reinterpret_cast<float4*>(dst + i) = make_float4(v[i] * p.scale_log2, v[i + 1] * p.scale_log2,
+                                                                v[i + 2] * p.scale_log2, v[i + 3] * p.scale_log2);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (key0 + c * 32 + i < L) dst[i] = v[i] * p.scale_log2;
+          }
+        }
+        float packed[16];
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          const float e0 = ex2(fmaf(v[i], p.scale_log2, neg_ref));      // exp2(-inf) = 0 for a masked key
+          const float e1 = ex2(fmaf(v[i + 1], p.scale_log2, neg_ref));
+          ls[i & 2] += e0;
+          ls[(i & 2) + 1] += e1;
+          packed[i / 2] = __uint_as_float(pack_bf16(e0, e1));
+        }
+        tmem_st_32x16(s_addr + c * 16, packed);
       }
       l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-      tmem_st_32x32(lane_addr + 384 + s * 64 + half * (HN / 2), packed);
       tmem_wait_st();
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->p_full[s]);
+      if (lane == 0) mbar_arrive(&bars->p_full[x]);
     }
-    // the finished row: the halves' sums meet, O / l -> bf16, each half its own columns
-    const int xb = n_tiles & 1;                           // the exchange buffer the last tile did not use
-    xch[(xb * 2 + half) * kBM + r] = l;
-    pair_sync();
-    l += xch[(xb * 2 + (half ^ 1)) * kBM + r];
-    if (ok) ok = mbar_wait_bounded(&bars->o_done, 0, abort_flag, p.hdr, SITE_ATTN_ODONE, limit);
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
-      tc_fence_after_sync();
-      const float inv_l = 1.0f / l;
-      uint8_t* const orow = reinterpret_cast<uint8_t*>(p.out) +
-                            (static_cast<size_t>(row0 + t) * p.out_stride_tok + static_cast<size_t>(h) * p.out_stride_head) * 2 +
-                            half * D;                      // D / 2 elements of 2 bytes
+    if (nk > 0) {
+      // the finished row: the halves' sums meet, O / l -> bf16, each half its own columns
+      const int xb = nk & 1;                              // the exchange buffer the last tile did not use
+      xch[(xb * 2 + half) * kBM + r] = l;
+      pair_sync();
+      l += xch[(xb * 2 + (half ^ 1)) * kBM + r];
+      if (ok) ok = mbar_wait_bounded(&bars->o_done[x], 0, abort_flag, p.hdr, SITE_ATTN_ODONE, limit);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        tc_fence_after_sync();
+        const float inv_l = 1.0f / l;
+        uint8_t* const orow = reinterpret_cast<uint8_t*>(p.out) +
+                              (static_cast<size_t>(row0 + t) * p.out_stride_tok + static_cast<size_t>(h) * p.out_stride_head) * 2 +
+                              half * D;                      // D / 2 elements of 2 bytes
 #pragma unroll
-      for (int c = 0; c < D / 64; ++c) {
-        float o[32];
-        tmem_ld_32x32(lane_addr + 256 + half * (D / 2) + c * 32, o);
-        if (t < L) {
+        for (int c = 0; c < D / 64; ++c) {
+          float o[32];
+          tmem_ld_32x32(o_addr + c * 32, o);
+          if (t < L) {
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            uint4 w4;
-            w4.x = pack_bf16(o[u * 8 + 0] * inv_l, o[u * 8 + 1] * inv_l);
-            w4.y = pack_bf16(o[u * 8 + 2] * inv_l, o[u * 8 + 3] * inv_l);
-            w4.z = pack_bf16(o[u * 8 + 4] * inv_l, o[u * 8 + 5] * inv_l);
-            w4.w = pack_bf16(o[u * 8 + 6] * inv_l, o[u * 8 + 7] * inv_l);
-            *reinterpret_cast<uint4*>(orow + c * 64 + u * 16) = w4;
+            for (int u = 0; u < 4; ++u) {
+              uint4 w4;
+              w4.x = pack_bf16(o[u * 8 + 0] * inv_l, o[u * 8 + 1] * inv_l);
+              w4.y = pack_bf16(o[u * 8 + 2] * inv_l, o[u * 8 + 3] * inv_l);
+              w4.z = pack_bf16(o[u * 8 + 4] * inv_l, o[u * 8 + 5] * inv_l);
+              w4.w = pack_bf16(o[u * 8 + 6] * inv_l, o[u * 8 + 7] * inv_l);
+              *reinterpret_cast<uint4*>(orow + c * 64 + u * 16) = w4;
+            }
           }
         }
+        if (is_window && half == 0) p.wstat[(static_cast<size_t>(b) * p.n_q_heads + h) * p.window + jw] = make_float2(m_ref, l);
       }
-      if (is_window && half == 0) p.wstat[(static_cast<size_t>(b) * p.n_q_heads + h) * p.window + jw] = make_float2(m_ref, l);
     }
   }
 
@@ -473,7 +505,7 @@ static cudaError_t launch_attn_t(const CUtensorMap& tq, const CUtensorMap& tk, c
     configured.set(dev);
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((max_len + kBM - 1) / kBM, p.n_q_heads, p.batch);
+  cfg.gridDim = dim3((max_len + 2 * kBM - 1) / (2 * kBM), p.n_q_heads, p.batch);
   cfg.blockDim = dim3(kAttnThreads);
   cfg.dynamicSmemBytes = Cfg::kSmemBytes;
   cfg.stream = stream;

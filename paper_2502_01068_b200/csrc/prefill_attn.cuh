@@ -16,7 +16,7 @@ struct PrefillParams {
   float2* wstat;              // [batch][n_q_heads][window]: (reference, sum of exp2(s - reference)) of the window rows
   WorkspaceHeader* hdr;
   long long wait_limit;
-  int skip_commit_tile;       // test hook: the issuer does not signal that P of this key tile was consumed (-1: none)
+  int skip_commit_tile;       // test hook: the first query tile's issuer does not signal that S of this key tile is ready (-1: none)
 };
 
 struct WindowScoresParams {

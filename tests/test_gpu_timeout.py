@@ -44,13 +44,16 @@ def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_correct(debug_hoo
     np.testing.assert_allclose(s_kv.cpu().numpy(), o["S_kv"], rtol=2e-3, atol=1e-12)
 
 
-SITE_ATTN_P_CONSUMED_WAIT = 34       # the softmax warps' wait for "P of the tile two before was consumed"
+SITE_ATTN_S_READY_WAIT = 33          # the softmax warps' wait for "S of this key tile is in tensor memory"
 SITE_ATTN_P_READY_WAIT = 31          # the issuer's wait for the P the stalled softmax warps never hand over
+SITE_ATTN_TURN_WAIT = 32             # the other query tile's issuer's wait for its turn, which the stalled one never passes on
+SITE_ATTN_RING_WAIT = 26             # the producer's wait for a K / V stage the stalled issuer never releases
 
 
 def test_prefill_attention_wait_that_runs_out(debug_hooks):
-    """The prefill attention's softmax warps wait (bounded) for the tensor core to have consumed P of the tile two
-    before; the test hook withholds that signal for one key tile.  The wait gives up after about two milliseconds,
+    """The prefill attention's softmax warps wait (bounded) for the tensor core to have left S of the key tile in
+    tensor memory; the test hook withholds that signal for one key tile of every CTA's first query tile.  The wait
+    gives up after about two milliseconds,
     every role of the CTA runs out of its loops, copies and contractions in flight are waited for, the status word
     says where -- and the next call on the same workspace is correct."""
     import oracle
@@ -65,11 +68,11 @@ def test_prefill_attention_wait_that_runs_out(debug_hooks):
     out = torch.zeros((L, wl.n_q_heads, wl.head_dim), dtype=torch.int16, device="cuda")
     s_kv = torch.zeros((wl.n_kv_heads, L), dtype=torch.float32, device="cuda")
     debug_hooks("wait_limit_cycles", 1 << 22)
-    debug_hooks("prefill_skip_commit", 2)                      # key tile 1: query tiles with four or more key tiles stall
+    debug_hooks("prefill_skip_commit", 2)                      # key tile 1: every CTA whose first query tile has two or more key tiles stalls
     B.fastkv_prefill_attention(shape, dev(q_full), dev(x.k), dev(x.v), out, s_kv, None, ws)
     status, site = B.fastkv_device_status(ws)
     assert status == B.ERR_DEVICE_TIMEOUT
-    assert site in (SITE_ATTN_P_CONSUMED_WAIT, SITE_ATTN_P_READY_WAIT)       # whichever of the two polls longer first
+    assert site in (SITE_ATTN_S_READY_WAIT, SITE_ATTN_P_READY_WAIT, SITE_ATTN_TURN_WAIT, SITE_ATTN_RING_WAIT)   # whichever gives up first
 
     debug_hooks("wait_limit_cycles", 0)
     debug_hooks("prefill_skip_commit", 0)
