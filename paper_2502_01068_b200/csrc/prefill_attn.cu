@@ -2,24 +2,31 @@
 // (Alg. 1: the TSP layer's own attention produces Att_l; Sec. 4.2 / App. D.4: the token importance
 // estimation is otherwise a separate pass over Q_window x K).
 //
-// One CTA per (128-query tile, query head); it walks the key tiles 0 .. tile of its last query:
+// One CTA per (pair of 128-query tiles A and B, query head); it walks the key tiles 0 .. tile of its last query:
 //
-//   producer   one thread: the Q tile once, then K and V tiles into two-stage rings by TMA;
-//   issuer     one thread: S = Q K^T (tcgen05.mma, 128 x 128 x d, fp32 in tensor memory, two S buffers so
-//              that the contraction of tile j+1 runs while tile j is in the softmax), then
-//              O += P V with P (bf16, packed two keys per column) read from tensor memory and V as an
-//              MN-major operand from shared memory (the V tile is used as TMA delivers it, keys x d
-//              with d contiguous).  With 128 x 128 tiles both operands of a contraction in shared
-//              memory would need all of its bandwidth (8 KB per 64 cycles), and K / V arrive and P would
-//              be written there as well: keeping P in tensor memory is what lets the tensor pipe run;
-//   softmax    eight warps, two threads per query row (tensor-memory lane = row; the two warps that
-//              share a lane quarter take 64 keys of the tile each and exchange their maxima through
-//              shared memory at one named barrier per tile): online softmax in log2 units with a
-//              lazily raised reference (the row's reference moves, and its O row is rescaled, only
-//              when a logit exceeds it by more than 8 binary orders of magnitude), P rounded to bf16
-//              and stored to tensor memory (two buffers), and at the end O / l -> bf16 -> global memory.
+//   producer   one thread: the two Q tiles once, then K and V tiles into two-stage rings by TMA (both query
+//              tiles use every K / V tile: half the shared-memory fills per flop);
+//   issuers    one warp per query tile (on two warp schedulers: issuing a contraction holds up the other warps
+//              of the issuer's scheduler), walking its loop as a whole warp with one elected lane per
+//              instruction.  Per key tile j a tile's issuer issues one block: O += P_(j-1) V_(j-1) with P (bf16,
+//              packed two keys per column) read from tensor memory and V as an MN-major operand from shared
+//              memory (the V tile is used as TMA delivers it, keys x d with d contiguous), then S = Q K_j^T
+//              (tcgen05.mma, 128 x 128 x d, fp32 in tensor memory).  Contractions of one thread execute in order,
+//              so S_j overwrites the tile's S / P columns only after the contraction that read P_(j-1) from
+//              them, and the softmax of key tile j finds O complete up to j - 1 -- no barrier for either.  The
+//              two tiles' blocks alternate on the tensor cores (A(0) B(0) A(1) B(1) ..., a turn barrier each
+//              way), which keeps the two softmaxes half a period apart: one tile's exponentials run under the
+//              other's contractions.  Left alone the two tiles fall into step and take turns waiting;
+//   softmax    eight warps per query tile, two threads per query row (tensor-memory lane = row; the two warps
+//              that share a lane quarter take 64 keys of the tile each and exchange their maxima through
+//              shared memory at one named barrier per tile): online softmax in log2 units with a lazily raised
+//              reference (the row's reference moves, and its O row is rescaled, only when a logit exceeds it by
+//              more than 8 binary orders of magnitude).  The logits stay in tensor memory and are read twice,
+//              32 at a time (maximum, then exponentials): 96 registers per thread let 19 warps share the SM.
+//              P is rounded to bf16 and stored into the first half of the thread's own S columns (columns it
+//              has read already); at the end O / l -> bf16 -> global memory.
 //
-// Tensor memory (512 columns): S buffers at 0 and 128, O at 256, P buffers (64 columns each) at 384 and 448.
+// Tensor memory (512 columns): S (and P inside it) of tile A at 0, of tile B at 128; O of A at 256, of B at 256 + d.
 //
 // The by-product: the threads whose query row is one of the last w of its sequence (the observation
 // window) also store their scaled logits of every key (fp32, log2 units) and, at the end, their
