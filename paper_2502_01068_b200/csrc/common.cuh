@@ -156,6 +156,25 @@ __device__ __forceinline__ bool mbar_wait_parked(uint64_t* bar, uint32_t parity,
   }
 }
 
+// The wait of an issuing warp whose wake-up is on the critical path: a suspended thread (above) resumes some
+// 0.5 kcycles after the phase completes; a poll every ~50 ns answers within ~0.1 kcycles and still leaves the
+// scheduler's issue slots to the compute warps.  Bounded like every other wait.
+__device__ __forceinline__ bool mbar_wait_nap(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                              WorkspaceHeader* hdr, int site, long long limit) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+    __nanosleep(50);
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > limit) {
+      *abort_flag = 1;
+      raise_status(hdr, FASTKV_ERR_DEVICE_TIMEOUT, site);
+      return false;
+    }
+  }
+}
+
 // The wait a role uses for its own copies or contractions still in flight before it leaves: bounded
 // like every other wait, but it does not give up just because the CTA is aborting.
 __device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity, WorkspaceHeader* hdr, int site,

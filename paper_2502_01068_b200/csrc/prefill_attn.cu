@@ -213,7 +213,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     // O += P V (1), ...: S of the next key tile overwrites the tile's S / P columns only after the contraction that
     // read P from them, and the softmax of key tile j finds O complete up to j - 1, with no barrier for either.
     // The two tiles' issuers sit on two warp schedulers (issuing a contraction holds up the other warps of the
-    // issuer's scheduler); each walks its loop as a whole warp, one elected lane issues.
+    // issuer's scheduler); each walks its loop as a whole warp, one elected lane issues; its waits poll every ~50 ns
+    // (a hot polling loop takes the scheduler's issue slots, a suspended wait wakes 0.5 kcycles late).
     const int x = warp - 1;
     const int nk = x == 0 ? n_key_a : n_key_b;
     constexpr uint32_t idesc_s = umma_idesc_bf16_f32(kBM, kBN);
@@ -224,7 +225,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     int committed = 0;
     auto first = [&](int j) {                              // S = Q K_j^T
       const int ks = j % NS;
-      ok = mbar_wait_parked(&bars->k_full[ks], (j / NS) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit);
+      ok = mbar_wait_nap(&bars->k_full[ks], (j / NS) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) return;
       tc_fence_after_sync();
@@ -254,7 +255,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       ++committed;
     };
     if (nk > 0) {
-      ok = mbar_wait_parked(&bars->q_full, 0, abort_flag, p.hdr, SITE_ATTN_Q, limit);
+      ok = mbar_wait_nap(&bars->q_full, 0, abort_flag, p.hdr, SITE_ATTN_Q, limit);
       ok = __all_sync(0xffffffffu, ok);
     }
     // Block jb of a tile = [O += P V of key tile jb - 1] [S of key tile jb].  The two tiles' blocks alternate on the
@@ -264,14 +265,14 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     int jb = 0;
     for (; nk > 0 && jb <= nk && ok; ++jb) {
       if (jb > 0) {
-        ok = mbar_wait_parked(&bars->v_full[(jb - 1) % NS], ((jb - 1) / NS) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit) &&
-             mbar_wait_parked(&bars->p_full[x], (jb - 1) & 1, abort_flag, p.hdr, SITE_ATTN_P, limit);
+        ok = mbar_wait_nap(&bars->v_full[(jb - 1) % NS], ((jb - 1) / NS) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit) &&
+             mbar_wait_nap(&bars->p_full[x], (jb - 1) & 1, abort_flag, p.hdr, SITE_ATTN_P, limit);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
       }
       if (b_active) {
-        if (x == 0 && jb >= 1) ok = mbar_wait_parked(&bars->turn[0], (jb - 1) & 1, abort_flag, p.hdr, SITE_ATTN_S, limit);
-        if (x == 1 && jb <= n_key_a) ok = mbar_wait_parked(&bars->turn[1], jb & 1, abort_flag, p.hdr, SITE_ATTN_S, limit);
+        if (x == 0 && jb >= 1) ok = mbar_wait_nap(&bars->turn[0], (jb - 1) & 1, abort_flag, p.hdr, SITE_ATTN_S, limit);
+        if (x == 1 && jb <= n_key_a) ok = mbar_wait_nap(&bars->turn[1], jb & 1, abort_flag, p.hdr, SITE_ATTN_S, limit);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
       }
@@ -285,11 +286,11 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     // the stage still counts two releases
     for (int jj = (nk == 0 || all_issued) ? nk : n_tiles; jj < n_tiles; ++jj) {
       const int s = jj % NS;
-      bool fine = mbar_wait_parked(&bars->k_full[s], (jj / NS) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit);
+      bool fine = mbar_wait_nap(&bars->k_full[s], (jj / NS) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit);
       fine = __all_sync(0xffffffffu, fine);
       if (!fine) break;
       if (lane == 0) mbar_arrive(&bars->k_empty[s]);
-      fine = mbar_wait_parked(&bars->v_full[s], (jj / NS) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit);
+      fine = mbar_wait_nap(&bars->v_full[s], (jj / NS) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit);
       fine = __all_sync(0xffffffffu, fine);
       if (!fine) break;
       if (lane == 0) mbar_arrive(&bars->v_empty[s]);
