@@ -324,6 +324,8 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 
   if (warp == 0) {
     // ---------------- producer: K tiles (and the phase's query rows) by TMA ----------------
+    // (the producer and the issuer wait with a poll every ~50 ns: a hot polling loop takes issue slots from the
+    //  pass-1 warps on their schedulers)
     if (lane == 0) {
       const uint64_t pol_k = l2_policy_evict_first();      // K is read exactly once
       const uint64_t pol_q = l2_policy_evict_last();
@@ -334,7 +336,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
       while (ok && next_phase<PART>(p, pit, cta, ncta, part_tab, w)) {
         if (w.n == 0) continue;
         const int h = u & 1;
-        if (u >= 2) ok = mbar_wait_bounded(&bars->q_empty[h], ((u >> 1) - 1) & 1, abort_flag, p.hdr, SITE_FUSED_Q_EMPTY, limit);
+        if (u >= 2) ok = mbar_wait_nap(&bars->q_empty[h], ((u >> 1) - 1) & 1, abort_flag, p.hdr, SITE_FUSED_Q_EMPTY, limit);
         if (!ok) break;
         const int q_row0 = (p.q_layout == FASTKV_Q_WINDOW) ? w.b * p.window : w.row0 + w.L - p.window;
         mbar_arrive_expect_tx(&bars->q_full[h], Cfg::KH * p.n_rows * 128);
@@ -344,7 +346,7 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         ++uq;
         for (int i = 0; i < w.n; ++i, ++T) {
           const int s = T % kStages;
-          ok = mbar_wait_bounded(&bars->empty[s], ((T / kStages) & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_EMPTY, limit);
+          ok = mbar_wait_nap(&bars->empty[s], ((T / kStages) & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_EMPTY, limit);
           if (!ok) break;
           mbar_arrive_expect_tx(&bars->full[s], Cfg::kStageBytes);
           for (int c = 0; c < Cfg::KH; ++c)
@@ -375,13 +377,13 @@ score_parked_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
       while (ok && next_phase<PART>(p, pit, cta, ncta, part_tab, w)) {
         if (w.n == 0) continue;
         const int h = u & 1;
-        ok = mbar_wait_bounded(&bars->q_full[h], (u >> 1) & 1, abort_flag, p.hdr, SITE_FUSED_Q_FULL, limit);
+        ok = mbar_wait_nap(&bars->q_full[h], (u >> 1) & 1, abort_flag, p.hdr, SITE_FUSED_Q_FULL, limit);
         if (!ok) break;
         const uint32_t q_addr = smem_u32(smem_q + h * Cfg::kQBytes);
         for (int i = 0; i < w.n; ++i, ++T) {
           const int s = T % kStages, a = T % kSlots;
-          ok = mbar_wait_bounded(&bars->slot_free[a], ((T / kSlots) & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_ACC_FREE, limit) &&
-               mbar_wait_bounded(&bars->full[s], (T / kStages) & 1, abort_flag, p.hdr, SITE_FUSED_FULL, limit);
+          ok = mbar_wait_nap(&bars->slot_free[a], ((T / kSlots) & 1) ^ 1, abort_flag, p.hdr, SITE_FUSED_ACC_FREE, limit) &&
+               mbar_wait_nap(&bars->full[s], (T / kStages) & 1, abort_flag, p.hdr, SITE_FUSED_FULL, limit);
           if (!ok) break;
           tc_fence_after_sync();
           const uint32_t k_addr = smem_u32(smem_k + s * Cfg::kStageBytes);
