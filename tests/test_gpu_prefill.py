@@ -107,3 +107,27 @@ def test_peaked_and_wide_logits():
     ref = oracle.prefill_attention(q_full, x.k, x.v, scale=2.0)
     err = np.abs(got - ref)
     assert np.all(err <= O_RTOL * np.abs(ref) + O_ATOL), float(err.max())
+
+
+def test_long_prompts_on_sampled_rows():
+    """Prompts of tens of key tiles (a single one that ends 77 tokens into a pair of query tiles, and a ragged
+    batch): the oracle of the whole attention would take minutes, so sampled query rows -- the first rows, rows on
+    both sides of the 128- and 256-row boundaries, rows deep in the prompt and the last rows -- are checked one by
+    one against the oracle of a single query over its causal prefix (oracle.decode_attention: the same softmax
+    attention of one token over keys 0 .. t)."""
+    for lens, Hq, Hkv, d in (([16384 + 77], 8, 2, 128), ([5000, 129, 9000], 4, 1, 64)):
+        wl = small("prefill_long", 990 + len(lens), lens, Hq=Hq, Hkv=Hkv, d=d)
+        x = W.make_layer(wl)
+        q_full = W.full_q(wl, x)
+        got, _, _ = run_prefill(wl, x, q_full, want_scores=False)
+        cu = x.cu_seqlens
+        rng = np.random.default_rng(5)
+        for b, L in enumerate(lens):
+            a = int(cu[b])
+            rows = {0, 1, 127, 128, 129, 255, 256, 257, 383, 384, L - 1, L - 2, L - 130} | set(int(t) for t in rng.integers(0, L, 12))
+            for t in sorted(r for r in rows if 0 <= r < L):
+                kc = np.ascontiguousarray(x.k[a:a + t + 1].transpose(1, 0, 2))     # [Hkv, t + 1, d]
+                vc = np.ascontiguousarray(x.v[a:a + t + 1].transpose(1, 0, 2))
+                ref, _ = oracle.decode_attention(q_full[a + t], kc, vc)
+                err = np.abs(got[a + t] - ref)
+                assert np.all(err <= O_RTOL * np.abs(ref) + O_ATOL), (lens, b, t, float(err.max()))
