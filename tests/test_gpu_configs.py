@@ -60,3 +60,30 @@ def test_llama8b_32k_sweep():
             if np.array_equal(g["idx_tsp"], o["idx_tsp"]):
                 np.testing.assert_array_equal(pos_g, pos_o)
     print("sweep: boundary flips over 32 layers: %d" % flips)
+
+
+def test_llama8b_128k_prefill_attention_hands_out_the_layer_scores():
+    """The 131072-token layer through the prefill attention in the launch configuration the bench times: the
+    scores it hands out against the oracle of the scoring path (2e-3 relative, as for fastkv_score), and the
+    attention output on sampled rows against the oracle of one query over its causal prefix."""
+    import oracle
+    from tests.test_gpu_prefill import O_ATOL, O_RTOL, run_prefill
+    wl = W.llama8b_128k()
+    x = W.make_layer(wl, with_hidden=False)
+    q_full = W.full_q(wl, x)
+    got, s_kv, s_tsp = run_prefill(wl, x, q_full)
+    o = oracle_layer(wl, x, do_compact=False)
+    np.testing.assert_allclose(s_kv, o["S_kv"], rtol=2e-3, atol=1e-12)
+    np.testing.assert_allclose(s_tsp, o["S_tsp"], rtol=2e-3, atol=1e-12)
+    L = wl.total_len
+    rng = np.random.default_rng(9)
+    rows = sorted({0, 255, 256, L // 2, L - 257, L - 256, L - 9, L - 1} | set(int(t) for t in rng.integers(0, L, 6)))
+    worst = 0.0
+    for t in rows:
+        kc = np.ascontiguousarray(x.k[:t + 1].transpose(1, 0, 2))
+        vc = np.ascontiguousarray(x.v[:t + 1].transpose(1, 0, 2))
+        ref, _ = oracle.decode_attention(q_full[t], kc, vc)
+        err = np.abs(got[t] - ref)
+        worst = max(worst, float(err.max()))
+        assert np.all(err <= O_RTOL * np.abs(ref) + O_ATOL), (t, float(err.max()))
+    print("128k prefill attention: worst abs output error on %d sampled rows %.3e" % (len(rows), worst))
