@@ -7,7 +7,8 @@
 // rate; so they run as warp-level m16n8k16 bf16 tensor-core products, whose only job here is to cut the
 // instruction count (~7 per kept entry).
 //
-// Split-KV: one CTA per (key range, KV head, sequence), and inside the CTA every warp works on its own: it
+// Split-KV: one CTA (eight warps; four for batches with more pairs than SMs) per (key range, KV head, sequence), and
+// inside the CTA every warp works on its own: it
 // owns a ring of shared-memory stages (16 kept entries of K and of V each) that one lane fills with tiled
 // TMA copies (boxes of 16 rows x 64 elements in the 128-byte swizzle, which makes the 8x8 matrix loads
 // conflict-free; one bulk copy per padded row instead was bound by the ~100 cycles each copy takes to
@@ -24,8 +25,8 @@ namespace fastkv {
 namespace {
 
 constexpr int kDecStages = 3;       // stages per warp: two chunks in flight while one is consumed
-constexpr int kDecWarps = 8;
-constexpr int kDecThreads = 32 * kDecWarps;
+// Warps per CTA: 8 (one CTA per SM) when the launch has fewer (key range, KV head, sequence) triples than SMs can hold
+// that way, 4 (two CTAs per SM) for batches with more pairs than that: the launch then runs as one wave.
 constexpr int kDecChunk = 16;       // kept entries per stage: the K extent of the second product
 constexpr int kDecHeads = 8;        // query heads per KV head, padded: the N extent of the second product
 
@@ -54,7 +55,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return r;
 }
 
-template <int D>
+template <int D, int kDecWarps>
 struct DecCfg {
   static constexpr int kBoxes = D / 64;                               // 64-element (128-byte) column blocks of a row
   static constexpr int kBoxBytes = kDecChunk * 128;                   // one box: 16 rows x 128 bytes, swizzled
@@ -67,10 +68,11 @@ struct DecCfg {
 
 }  // namespace
 
-template <int D>
-__global__ void __launch_bounds__(kDecThreads)
+template <int D, int kDecWarps>
+__global__ void __launch_bounds__(32 * kDecWarps)
 decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const DecodeParams p) {
-  using Cfg = DecCfg<D>;
+  using Cfg = DecCfg<D, kDecWarps>;
+  constexpr int kDecThreads = 32 * kDecWarps;
   constexpr int KS = D / 16;                    // 16-wide steps over the head dimension (first product)
   constexpr int MT = D / 16;                    // 16-row tiles of the head dimension (second product)
   extern __shared__ uint8_t smem_raw[];
@@ -303,10 +305,11 @@ size_t decode_workspace_bytes(int batch, int n_kv_heads, int group, int head_dim
   return sizeof(WorkspaceHeader) + (parts * sizeof(float2) + 255) / 256 * 256 + parts * head_dim * sizeof(float);
 }
 
-template <int D>
-static cudaError_t launch_decode_d(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, int batch, int k_max,
-                                   cudaStream_t stream, int* launches) {
-  constexpr int kSmem = DecCfg<D>::kSmem;
+template <int D, int kDecWarps>
+static cudaError_t launch_decode_w(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, int batch, int k_max,
+                                   cudaStream_t stream, int* launches, int* capacity_out) {
+  constexpr int kSmem = DecCfg<D, kDecWarps>::kSmem;
+  constexpr int kDecThreads = 32 * kDecWarps;
   // launch attributes and occupancy are per device: cached by device ordinal
   static PerDeviceOnce configured;
   static int capacity_of[PerDeviceOnce::kMaxDevices];
@@ -315,24 +318,28 @@ static cudaError_t launch_decode_d(const CUtensorMap& tk, const CUtensorMap& tv,
   if (e0 != cudaSuccess) return e0;
   if (dev < 0 || dev >= PerDeviceOnce::kMaxDevices) return cudaErrorInvalidDevice;
   if (!configured.done(dev)) {
-    cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<D, kDecWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     // one wave: as many splits as keep every CTA resident at once
     int sms = 148, per_sm = 1;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_attn_kernel<D>, kDecThreads, kSmem) != cudaSuccess || per_sm < 1)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_attn_kernel<D, kDecWarps>, kDecThreads, kSmem) != cudaSuccess || per_sm < 1)
       per_sm = 1;
     capacity_of[dev] = sms * per_sm;
     configured.set(dev);
   }
   const int capacity = capacity_of[dev];
+  if (capacity_out != nullptr) {                 // only asked how many CTAs this shape of CTA keeps resident
+    *capacity_out = capacity;
+    return cudaSuccess;
+  }
   int splits = capacity / (batch * p.n_kv_heads);
   const int chunks = (k_max + kDecChunk - 1) / kDecChunk;
   const int useful = (chunks + kDecWarps - 1) / kDecWarps;      // at least one chunk per warp
   if (splits > useful) splits = useful;
   if (splits > kDecodeMaxSplits) splits = kDecodeMaxSplits;
   if (splits < 1) splits = 1;
-  decode_attn_kernel<D><<<dim3(splits, p.n_kv_heads, batch), kDecThreads, kSmem, stream>>>(tk, tv, p);
+  decode_attn_kernel<D, kDecWarps><<<dim3(splits, p.n_kv_heads, batch), kDecThreads, kSmem, stream>>>(tk, tv, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   *launches = 1;
@@ -347,6 +354,17 @@ static cudaError_t launch_decode_d(const CUtensorMap& tk, const CUtensorMap& tv,
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, decode_combine_kernel<D>, static_cast<const DecodeParams&>(p), splits);
+}
+
+template <int D>
+static cudaError_t launch_decode_d(const CUtensorMap& tk, const CUtensorMap& tv, DecodeParams& p, int batch, int k_max,
+                                   cudaStream_t stream, int* launches) {
+  int big = 0;
+  cudaError_t e = launch_decode_w<D, 8>(tk, tv, p, batch, k_max, stream, launches, &big);
+  if (e != cudaSuccess) return e;
+  // more (KV head, sequence) pairs than one-CTA-per-SM holds: the small CTAs, two per SM, keep the launch in one wave
+  if (batch * p.n_kv_heads > big) return launch_decode_w<D, 4>(tk, tv, p, batch, k_max, stream, launches, nullptr);
+  return launch_decode_w<D, 8>(tk, tv, p, batch, k_max, stream, launches, nullptr);
 }
 
 cudaError_t launch_decode_attn(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, DecodeParams& p, int head_dim, int batch,
