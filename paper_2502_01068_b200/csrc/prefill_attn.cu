@@ -123,11 +123,17 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   float* xch_all = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 256);   // [tile][2][2][128]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b = blockIdx.z, h = blockIdx.y, g = h / p.group;
+  // Launch order (blockIdx.x fastest): when K and V of all heads fit in L2 together, all query heads fastest, then
+  // the pairs of query tiles, longest rows first -- every head's long CTAs start before anybody's short ones.  For
+  // long prompts the heads of one GQA group fastest, then the pairs, then the KV heads: what runs at the same time
+  // works on one or two KV heads' K and V, which stay in L2.
+  const int heads_x = static_cast<int>(gridDim.x);                 // n_q_heads or group
+  const int per_z = p.n_q_heads / heads_x;                         // 1 or n_kv_heads
+  const int b = blockIdx.z / per_z, h = (blockIdx.z - b * per_z) * heads_x + blockIdx.x, g = h / p.group;
   const int row0 = p.cu_seqlens ? p.cu_seqlens[b] : 0;
   const int L = p.cu_seqlens ? p.cu_seqlens[b + 1] - row0 : p.total_len;
   const int n_pairs = (L + 2 * kBM - 1) / (2 * kBM);
-  const int qp = n_pairs - 1 - static_cast<int>(blockIdx.x);       // the longest rows first
+  const int qp = n_pairs - 1 - static_cast<int>(blockIdx.y);       // the longest rows first
   if (qp < 0) return;                                              // (uniform per CTA, before any barrier)
   if (smem_u32(smem) & 1023u) {                                    // never seen; would garble every tile
     if (threadIdx.x == 0) raise_status(p.hdr, FASTKV_ERR_UNSUPPORTED, SITE_ATTN_Q);
@@ -513,7 +519,11 @@ static cudaError_t launch_attn_t(const CUtensorMap& tq, const CUtensorMap& tk, c
     configured.set(dev);
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((max_len + 2 * kBM - 1) / (2 * kBM), p.n_q_heads, p.batch);
+  const int n_kv_heads = p.n_q_heads / p.group;
+  const long long kv_bytes = 2ll * p.total_len * n_kv_heads * D * 2;           // K and V of every head
+  const bool all_heads_first = kv_bytes <= (64ll << 20);                       // they stay in L2 whatever runs together
+  cfg.gridDim = all_heads_first ? dim3(p.n_q_heads, (max_len + 2 * kBM - 1) / (2 * kBM), p.batch)
+                                : dim3(p.group, (max_len + 2 * kBM - 1) / (2 * kBM), p.batch * n_kv_heads);
   cfg.blockDim = dim3(kAttnThreads);
   cfg.dynamicSmemBytes = Cfg::kSmemBytes;
   cfg.stream = stream;
