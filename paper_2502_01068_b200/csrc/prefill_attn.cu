@@ -229,12 +229,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     const uint32_t s_tmem = tmem_base + x * kBN, o_tmem = tmem_base + 256 + x * D;
     bool ok = true;
     int committed = 0;
-    auto first = [&](int j) {                              // S = Q K_j^T
+    auto first = [&](int j) {                              // S = Q K_j^T (the caller has seen K_j arrive)
       const int ks = j % NS;
-      ok = mbar_wait_nap(&bars->k_full[ks], (j / NS) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) return;
-      tc_fence_after_sync();
       const uint64_t a0 = umma_desc_k_sw128(q_addr), b0 = umma_desc_k_sw128(smem_u32(sK + ks * Cfg::kTileBytes));
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk) {                // 64-element chunk kk / 4, 32 bytes per step inside it
@@ -270,6 +266,11 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     // cores at the same time and the special-function unit at the same time, and each waits while the other works).
     int jb = 0;
     for (; nk > 0 && jb <= nk && ok; ++jb) {
+      if (jb < nk) {                                       // K of the block's S: long there when P arrives
+        ok = mbar_wait_nap(&bars->k_full[jb % NS], (jb / NS) & 1, abort_flag, p.hdr, SITE_ATTN_K, limit);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
       if (jb > 0) {
         ok = mbar_wait_nap(&bars->v_full[(jb - 1) % NS], ((jb - 1) / NS) & 1, abort_flag, p.hdr, SITE_ATTN_V, limit) &&
              mbar_wait_nap(&bars->p_full[x], (jb - 1) & 1, abort_flag, p.hdr, SITE_ATTN_P, limit);
